@@ -1,0 +1,164 @@
+/*
+ * isopo.h - C ABI of the B200 (sm_100a) implementation of the ISOPO per-linear-layer path.
+ *
+ * ISOPO ("Isometric Policy Optimization") transforms, layer by layer inside one backward pass,
+ * the advantages of the B sequences of a ragged microbatch before they are contracted with the
+ * per-sequence log-probability gradients of the layer's weight.  For one linear layer with packed
+ * input activations X [T, d_in] and output gradients dY [T, d_out] (the backward pass is run on
+ * sum(log_prob) WITHOUT advantages; Algorithm 1 and Algorithm 2 of the paper) the path is
+ *
+ *     G_i  = sum_{t in sequence i} dY[t,:]^T X[t,:]          [d_out, d_in]   (Alg. 1/2, reduce loop)
+ *     K_ij = <G_i, G_j>                                       [B, B]          (Alg. 2, NTK; Sec. 3 K = J J^T)
+ *     c    = transform(K, A)                                  [B]             (Sec. 2.1, 2.3, Fig. 3, Sec. 3)
+ *     dW   = sum_i c_i G_i = (c_seq(t) * dY)^T X              [d_out, d_in]   (Alg. 1/2, accumulate)
+ *
+ * Conventions shared by every entry point
+ *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are ordinary
+ *     host memory.  The caller owns every buffer; the library never allocates or frees device memory.
+ *   - X and dY are row-major, contiguous, 16-byte aligned; row t is token t of the packed microbatch;
+ *     sequence i owns rows seq_offsets[i] .. seq_offsets[i+1]-1, with seq_offsets[0] = 0,
+ *     seq_offsets[B] = T and every length >= 1.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and the call returns without synchronising.  The three calls of one layer must be issued in
+ *     order on the same stream with the same workspace.
+ *   - The return value reports what the host can detect (bad arguments, unsupported shapes, a
+ *     workspace that is too small, a CUDA launch error).  Conditions found on the device are
+ *     written to `*info` (dev, int32), which the caller zeroes beforehand and reads after
+ *     synchronising the stream: 0 = ok; 1..B = the leading minor of that order of K + lambda*I is
+ *     not positive definite (interacting transform); ISOPO_INFO_TIMEOUT | id = a bounded wait inside
+ *     kernel `id` ran out.  The library only ever overwrites a zero `*info`.  When `*info` != 0 the
+ *     outputs are unspecified (but every access stayed in bounds).
+ *   - There is no CPU fallback and no global state; one GPU.
+ */
+#ifndef ISOPO_H_
+#define ISOPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ISOPO_API __attribute__((visibility("default")))
+#else
+#define ISOPO_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ISOPO_OK = 0,
+  ISOPO_ERR_INVALID_ARG = 1,  /* null pointer, bad size, bad offsets, misaligned buffer */
+  ISOPO_ERR_UNSUPPORTED = 2,  /* valid request that this build has no kernel for */
+  ISOPO_ERR_WORKSPACE = 3,    /* ws_bytes smaller than isopo_workspace_bytes(...) */
+  ISOPO_ERR_CUDA = 4          /* a CUDA runtime/driver call failed; see isopo_last_cuda_error() */
+} isopo_status;
+
+typedef enum {
+  ISOPO_F32 = 0,   /* X, dY float32; SIMT FFMA kernels, K accumulated in float64 */
+  ISOPO_BF16 = 1   /* X, dY bfloat16; tcgen05 tensor-core kernels, float32 accumulation */
+} isopo_dtype;
+
+typedef enum {
+  ISOPO_PATH_AUTO = 0,        /* cost model picks one of the two below (isopo_choose_path) */
+  ISOPO_PATH_GRAM = 1,        /* K from token Grams, never forms G_i */
+  ISOPO_PATH_MATERIALISE = 2  /* forms every G_i in the workspace, K from them, dW from them */
+} isopo_path;
+
+typedef enum {
+  ISOPO_VAR_REINFORCE = 0,      /* c_i = A_i */
+  ISOPO_VAR_NORMALISED = 1,     /* c_i = A_i / sqrt(F_i^2 + lambda)           Sec. 2.1 display; Fig. 3 p = -1 */
+  ISOPO_VAR_DIRECTION = 2,      /* c_i = A_i / (F_i^2 / K_ii + lambda)        Sec. 2.3 display; Fig. 3 r = -2 */
+  ISOPO_VAR_EUCLID = 3,         /* c_i = A_i / sqrt(K_ii + lambda)            Fig. 3 q = -1 */
+  ISOPO_VAR_GENERAL = 4,        /* Fig. 3 with free p, q, r and three absolute regularisers */
+  ISOPO_VAR_INTERACTING = 5,    /* (K + lambda I) c = A                       Sec. 3 display; Alg. 2 */
+  ISOPO_VAR_NORMALISED_RAW = 6  /* as NORMALISED with F_i^2 = (1/B) sum_j K_ij^2 (Eq. F-norm-basic as printed) */
+} isopo_variant;
+
+#define ISOPO_INFO_TIMEOUT 0x40000000
+
+/* Human-readable name of a status code (static storage, never NULL). */
+ISOPO_API const char* isopo_status_string(isopo_status s);
+
+/* Text of the last CUDA error seen by this thread inside the library (static storage). */
+ISOPO_API const char* isopo_last_cuda_error(void);
+
+/*
+ * Path that ISOPO_PATH_AUTO resolves to for these sizes.  The Gram route costs
+ * (d_in + d_out) * sum_i-over-token-pairs ~ (d_in + d_out) T^2 flops; the materialised route adds
+ * B^2 d_in d_out flops and three passes over B d_in d_out stored gradients to the plain dW GEMM
+ * (whose 2 T d_in d_out flops it re-uses).  Gram wins only for short sequences.
+ */
+ISOPO_API isopo_path isopo_choose_path(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B);
+
+/*
+ * Bytes of device workspace the three calls of one layer need for `path` (AUTO allowed).
+ * The workspace holds the device copy of the offsets, the token -> sequence map and, on the
+ * materialised path, all B per-sequence gradients (bf16 for ISOPO_BF16, float32 for ISOPO_F32)
+ * in a tile-blocked order private to the library.  It must be 1024-byte aligned.  Returns 0 for
+ * invalid sizes.
+ */
+ISOPO_API size_t isopo_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path path);
+
+/*
+ * isopo_layer_gram: K_ij = <G_i, G_j>  (Alg. 2 "make neural tangent kernel"; K = J J^T of Sec. 3).
+ *
+ * GRAM path: uses that each token gradient is the rank-one matrix dY_t x_t^T (Eq. one, Eq. two), so
+ *   K_ij = sum_{t in i, s in j} (dY_t . dY_s)(x_t . x_s): tiles of X X^T and dY dY^T are formed in
+ *   tensor memory, multiplied elementwise and segment-summed; no T x T matrix reaches memory.
+ * MATERIALISE path: forms G_i = dY_i^T X_i (Alg. 2 reduce loop) for every i into the workspace, then
+ *   K = G_flat G_flat^T.
+ *
+ *   X, dY            dev, [T, d_in] and [T, d_out] of `dtype`, row-major
+ *   seq_offsets_host host, int64 [B+1]; copied before the call returns
+ *   K                dev, float32 [B, B] row-major, overwritten; exactly symmetric on return
+ *   ws, ws_bytes     dev workspace, see isopo_workspace_bytes
+ *   info             dev int32, see above
+ * ISOPO_BF16 requires d_in and d_out to be multiples of 8; the bf16 MATERIALISE path requires B <= 256.
+ */
+ISOPO_API isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                              const int64_t* seq_offsets_host, int B, isopo_path path, float* K, void* ws,
+                              size_t ws_bytes, int32_t* info, void* cuda_stream);
+
+/*
+ * isopo_transform_advantages: advantages A -> coefficients c (dW = sum_i c_i G_i).
+ *
+ * With F_i^2 = sum_j K_ij^2 / sum_j K_jj (the Fisher norm of Eq. F-norm-basic evaluated with the B
+ * sequence gradients as samples and normalised by their summed squared norms as in
+ * Eq. formal-F-norm) the variants are those listed at isopo_variant.  ISOPO_VAR_GENERAL computes
+ *   c_i = A_i * reg2(F_i; g[3])^g[0] * reg2(sqrt(K_ii); g[4])^g[1] * reg2(F_i / sqrt(K_ii); g[5])^g[2],
+ *   reg2(v; reg) = sqrt(v^2 + reg + 1e-8)                                         (Fig. 3),
+ * with g = opt_pqr_regs = {p, q, r, reg_F, reg_G, reg_rel} (host, 6 floats; required for GENERAL,
+ * ignored otherwise; `lambda` is ignored for GENERAL).  ISOPO_VAR_INTERACTING factors K + lambda*I
+ * by Cholesky in shared memory (float32) and refines the solution with float64 residuals; it
+ * requires B <= 256 and reports a non-positive pivot k (1-based) as *info = k.
+ *
+ *   K       dev, float32 [B, B] row-major (as written by isopo_layer_gram)
+ *   A       dev, float32 [B]
+ *   lambda  absolute regulariser, >= 0 (the caller multiplies by its running mean if it wants a relative one)
+ *   coeffs  dev, float32 [B], overwritten
+ */
+ISOPO_API isopo_status isopo_transform_advantages(const float* K, const float* A, int B, isopo_variant variant, float lambda,
+                                        const float* opt_pqr_regs, float* coeffs, int32_t* info, void* cuda_stream);
+
+/*
+ * isopo_weight_grad: dW = beta * dW + sum_i coeffs[i] * G_i   (Alg. 1 "grad += advantages * rescaled
+ * gradient" and "mod.grad += grad"; Alg. 2 "stack(seq_grads) @ advantages_preconditioned").
+ *
+ * `path` must be the value given to isopo_layer_gram for this layer (AUTO resolves identically).
+ * MATERIALISE: streams the G_i left in the workspace by isopo_layer_gram.  GRAM: one GEMM over all
+ * tokens, dW = (coeffs[seq(t)] * dY)^T X, with the per-token scale folded into the operand.
+ *
+ *   coeffs  dev, float32 [B]
+ *   dW      dev, float32 [d_out, d_in] row-major (the layout of `grad_out.T @ act_in`)
+ *   beta    0 (overwrite) or 1 (accumulate into the existing gradient)
+ * Other arguments as for isopo_layer_gram; seq_offsets_host must hold the same offsets.
+ */
+ISOPO_API isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                               const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
+                               float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ISOPO_H_ */

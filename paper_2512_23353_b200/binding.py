@@ -1,0 +1,177 @@
+"""Thin ctypes binding of libisopo.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  torch is used for device memory and
+the current stream, nothing else.  Importing this module without a built library raises.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libisopo.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
+F32, BF16 = 0, 1
+PATH_AUTO, PATH_GRAM, PATH_MATERIALISE = 0, 1, 2
+(VAR_REINFORCE, VAR_NORMALISED, VAR_DIRECTION, VAR_EUCLID, VAR_GENERAL, VAR_INTERACTING,
+ VAR_NORMALISED_RAW) = range(7)
+INFO_TIMEOUT = 0x40000000
+
+EXPORTS = (
+    "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",
+    "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad",
+)
+
+
+class IsopoError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(what)
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2512_23353_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    c = ctypes
+    lib.isopo_status_string.restype = c.c_char_p
+    lib.isopo_status_string.argtypes = [c.c_int]
+    lib.isopo_last_cuda_error.restype = c.c_char_p
+    lib.isopo_last_cuda_error.argtypes = []
+    lib.isopo_choose_path.restype = c.c_int
+    lib.isopo_choose_path.argtypes = [c.c_int, c.c_int64, c.c_int, c.c_int, c.c_int]
+    lib.isopo_workspace_bytes.restype = c.c_size_t
+    lib.isopo_workspace_bytes.argtypes = [c.c_int, c.c_int64, c.c_int, c.c_int, c.c_int, c.c_int]
+    lib.isopo_layer_gram.restype = c.c_int
+    lib.isopo_layer_gram.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
+                                     c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.isopo_transform_advantages.restype = c.c_int
+    lib.isopo_transform_advantages.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
+                                               c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.isopo_weight_grad.restype = c.c_int
+    lib.isopo_weight_grad.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
+                                      c.c_void_p, c.c_int, c.c_int, c.c_void_p, c.c_float, c.c_void_p, c.c_size_t,
+                                      c.c_void_p, c.c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        name = lib.isopo_status_string(status).decode()
+        extra = f" [{lib.isopo_last_cuda_error().decode()}]" if status == ERR_CUDA else ""
+        raise IsopoError(status, f"{what}: {name}{extra}")
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _offsets(seq_offsets) -> np.ndarray:
+    off = np.ascontiguousarray(np.asarray(seq_offsets, dtype=np.int64))
+    if off.ndim != 1 or off.shape[0] < 2:
+        raise ValueError("seq_offsets must be a 1-D array of B+1 entries")
+    return off
+
+
+def isopo_choose_path(dtype: int, T: int, d_in: int, d_out: int, B: int) -> int:
+    return lib.isopo_choose_path(dtype, T, d_in, d_out, B)
+
+
+def isopo_workspace_bytes(dtype: int, T: int, d_in: int, d_out: int, B: int, path: int = PATH_AUTO) -> int:
+    return lib.isopo_workspace_bytes(dtype, T, d_in, d_out, B, path)
+
+
+def alloc_workspace(dtype: int, T: int, d_in: int, d_out: int, B: int, path: int = PATH_AUTO, device="cuda"):
+    """A torch uint8 buffer of the size the library asks for (torch's allocator aligns to 512 B; the
+    view returned starts on a 1024-byte boundary)."""
+    n = isopo_workspace_bytes(dtype, T, d_in, d_out, B, path)
+    if n == 0:
+        raise IsopoError(ERR_INVALID_ARG, "isopo_workspace_bytes: invalid sizes")
+    raw = torch.empty(n + 1024, dtype=torch.uint8, device=device)
+    shift = (-raw.data_ptr()) % 1024
+    return raw[shift:shift + n]
+
+
+def isopo_layer_gram(X: torch.Tensor, dY: torch.Tensor, seq_offsets, K: torch.Tensor, ws: torch.Tensor,
+                     info: torch.Tensor, path: int = PATH_AUTO) -> None:
+    off = _offsets(seq_offsets)
+    B = off.shape[0] - 1
+    assert X.is_cuda and dY.is_cuda and X.is_contiguous() and dY.is_contiguous() and X.dtype == dY.dtype
+    assert K.dtype == torch.float32 and K.is_contiguous() and K.numel() == B * B
+    assert info.dtype == torch.int32 and ws.dtype == torch.uint8
+    st = lib.isopo_layer_gram(X.data_ptr(), dY.data_ptr(), _dtype_code(X), X.shape[0], X.shape[1], dY.shape[1],
+                              off.ctypes.data, B, path, K.data_ptr(), ws.data_ptr(), ws.numel(), info.data_ptr(),
+                              _stream())
+    _check(st, "isopo_layer_gram")
+
+
+def isopo_transform_advantages(K: torch.Tensor, A: torch.Tensor, variant: int, lam: float, coeffs: torch.Tensor,
+                               info: torch.Tensor, pqr_regs=None) -> None:
+    B = A.numel()
+    assert K.dtype == torch.float32 and A.dtype == torch.float32 and coeffs.dtype == torch.float32
+    assert K.is_contiguous() and K.numel() == B * B and coeffs.numel() == B
+    g = None
+    if pqr_regs is not None:
+        g = np.ascontiguousarray(np.asarray(pqr_regs, dtype=np.float32))
+        assert g.shape == (6,)
+    st = lib.isopo_transform_advantages(K.data_ptr(), A.data_ptr(), B, variant, float(lam),
+                                        g.ctypes.data if g is not None else None, coeffs.data_ptr(),
+                                        info.data_ptr(), _stream())
+    _check(st, "isopo_transform_advantages")
+
+
+def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, seq_offsets, dW: torch.Tensor,
+                      ws: torch.Tensor, info: torch.Tensor, path: int = PATH_AUTO, beta: float = 0.0) -> None:
+    off = _offsets(seq_offsets)
+    B = off.shape[0] - 1
+    assert dW.dtype == torch.float32 and dW.is_contiguous() and dW.shape == (dY.shape[1], X.shape[1])
+    assert coeffs.dtype == torch.float32 and coeffs.numel() == B
+    st = lib.isopo_weight_grad(X.data_ptr(), dY.data_ptr(), _dtype_code(X), X.shape[0], X.shape[1], dY.shape[1],
+                               coeffs.data_ptr(), off.ctypes.data, B, path, dW.data_ptr(), float(beta),
+                               ws.data_ptr(), ws.numel(), info.data_ptr(), _stream())
+    _check(st, "isopo_weight_grad")
+
+
+@dataclass
+class LayerResult:
+    K: torch.Tensor
+    coeffs: torch.Tensor
+    dW: torch.Tensor
+    info: int
+
+
+def isopo_layer(X, dY, seq_offsets, A, variant, lam, path=PATH_AUTO, pqr_regs=None, ws=None) -> LayerResult:
+    """The three calls of one layer in order on the current stream; synchronises to read `info`."""
+    off = _offsets(seq_offsets)
+    B = off.shape[0] - 1
+    dev = X.device
+    dt = _dtype_code(X)
+    if ws is None:
+        ws = alloc_workspace(dt, X.shape[0], X.shape[1], dY.shape[1], B, path, dev)
+    K = torch.empty((B, B), dtype=torch.float32, device=dev)
+    c = torch.empty(B, dtype=torch.float32, device=dev)
+    dW = torch.empty((dY.shape[1], X.shape[1]), dtype=torch.float32, device=dev)
+    info = torch.zeros(1, dtype=torch.int32, device=dev)
+    isopo_layer_gram(X, dY, off, K, ws, info, path)
+    isopo_transform_advantages(K, A, variant, lam, c, info, pqr_regs)
+    isopo_weight_grad(X, dY, c, off, dW, ws, info, path, 0.0)
+    return LayerResult(K, c, dW, int(info.item()))

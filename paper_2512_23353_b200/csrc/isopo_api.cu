@@ -1,0 +1,172 @@
+// C-ABI entry points of libisopo: argument validation, workspace layout, path choice, dispatch.
+// Every step of the path runs in the CUDA kernels launched from here; there is no host arithmetic
+// on the data and no CPU fallback.
+#include <cstdio>
+#include <cstring>
+
+#include "isopo_internal.h"
+
+namespace isopo {
+
+static thread_local char g_cuda_err[256] = "no error";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
+}
+
+WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path resolved) {
+  WsLayout L{};
+  size_t p = 0;
+  L.off_offsets = p;
+  p = align_up(p + sizeof(int64_t) * (size_t)(B + 1), 1024);
+  L.off_tokseq = p;
+  p = align_up(p + sizeof(int32_t) * (size_t)T, 1024);
+  L.off_kacc = p;
+  if (dtype == ISOPO_F32) p = align_up(p + sizeof(double) * (size_t)B * (size_t)B, 1024);
+  L.off_G = p;
+  if (dtype == ISOPO_BF16) {
+    L.tiles_m = (d_out + kTileM - 1) / kTileM;
+    L.tiles_n = (d_in + kTileN - 1) / kTileN;
+    L.n_pad = (int64_t)L.tiles_m * L.tiles_n * kTileElems;
+    if (resolved == ISOPO_PATH_MATERIALISE) p = align_up(p + (size_t)2 * (size_t)B * (size_t)L.n_pad, 1024);
+  } else {
+    L.tiles_m = L.tiles_n = 0;
+    L.n_pad = (int64_t)d_in * d_out;
+    if (resolved == ISOPO_PATH_MATERIALISE) p = align_up(p + (size_t)4 * (size_t)B * (size_t)L.n_pad, 1024);
+  }
+  L.total = p;
+  return L;
+}
+
+static bool sizes_ok(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B) {
+  if (dtype != ISOPO_F32 && dtype != ISOPO_BF16) return false;
+  if (T < 1 || B < 1 || d_in < 1 || d_out < 1 || (int64_t)B > T) return false;
+  if (T > ((int64_t)1 << 31) - 1024) return false;  // token coordinates are 32-bit in the tensor maps
+  return true;
+}
+
+static isopo_status check_layer_args(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                                     const int64_t* off, int B, isopo_path path, const void* ws) {
+  if (!X || !dY || !off || !ws) return ISOPO_ERR_INVALID_ARG;
+  if (!sizes_ok(dtype, T, d_in, d_out, B)) return ISOPO_ERR_INVALID_ARG;
+  if (path != ISOPO_PATH_AUTO && path != ISOPO_PATH_GRAM && path != ISOPO_PATH_MATERIALISE)
+    return ISOPO_ERR_INVALID_ARG;
+  if (((uintptr_t)X & 15) || ((uintptr_t)dY & 15) || ((uintptr_t)ws & 1023)) return ISOPO_ERR_INVALID_ARG;
+  if (off[0] != 0 || off[B] != T) return ISOPO_ERR_INVALID_ARG;
+  for (int i = 0; i < B; ++i)
+    if (off[i + 1] <= off[i]) return ISOPO_ERR_INVALID_ARG;
+  if (dtype == ISOPO_BF16 && ((d_in & 7) || (d_out & 7))) return ISOPO_ERR_UNSUPPORTED;
+  return ISOPO_OK;
+}
+
+static isopo_path resolve_path(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path path) {
+  return path == ISOPO_PATH_AUTO ? isopo_choose_path(dtype, T, d_in, d_out, B) : path;
+}
+
+}  // namespace isopo
+
+using namespace isopo;
+
+extern "C" {
+
+const char* isopo_status_string(isopo_status s) {
+  switch (s) {
+    case ISOPO_OK: return "ISOPO_OK";
+    case ISOPO_ERR_INVALID_ARG: return "ISOPO_ERR_INVALID_ARG";
+    case ISOPO_ERR_UNSUPPORTED: return "ISOPO_ERR_UNSUPPORTED";
+    case ISOPO_ERR_WORKSPACE: return "ISOPO_ERR_WORKSPACE";
+    case ISOPO_ERR_CUDA: return "ISOPO_ERR_CUDA";
+  }
+  return "ISOPO_ERR_UNKNOWN";
+}
+
+const char* isopo_last_cuda_error(void) { return g_cuda_err; }
+
+isopo_path isopo_choose_path(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B) {
+  if (!sizes_ok(dtype, T, d_in, d_out, B)) return ISOPO_PATH_GRAM;
+  if (dtype == ISOPO_BF16 && B > 256) return ISOPO_PATH_GRAM;  // stored-gradient kernels hold all B rows on chip
+  // Modelled extra time over the plain dW GEMM (which both routes pay once).
+  const double peak = dtype == ISOPO_BF16 ? 1.39e15 : 4.0e13;  // flop/s: tcgen05 bf16 vs SIMT fp32
+  const double bw = 6.5e12;                                     // HBM bytes/s
+  const double elt = dtype == ISOPO_BF16 ? 2.0 : 4.0;
+  const double N = (double)d_in * (double)d_out;
+  const double t_gram = (double)(d_in + d_out) * (double)T * (double)T / peak;
+  const double t_mat = (double)B * (double)B * N / peak + 3.0 * elt * (double)B * N / bw;
+  return t_gram < t_mat ? ISOPO_PATH_GRAM : ISOPO_PATH_MATERIALISE;
+}
+
+size_t isopo_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path path) {
+  if (!sizes_ok(dtype, T, d_in, d_out, B)) return 0;
+  if (path != ISOPO_PATH_AUTO && path != ISOPO_PATH_GRAM && path != ISOPO_PATH_MATERIALISE) return 0;
+  return ws_layout(dtype, T, d_in, d_out, B, resolve_path(dtype, T, d_in, d_out, B, path)).total;
+}
+
+isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                              const int64_t* seq_offsets_host, int B, isopo_path path, float* K, void* ws,
+                              size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  if (!K || !info) return ISOPO_ERR_INVALID_ARG;
+  isopo_status s = check_layer_args(X, dY, dtype, T, d_in, d_out, seq_offsets_host, B, path, ws);
+  if (s != ISOPO_OK) return s;
+  const isopo_path rp = resolve_path(dtype, T, d_in, d_out, B, path);
+  if (dtype == ISOPO_BF16 && rp == ISOPO_PATH_MATERIALISE && B > 256) return ISOPO_ERR_UNSUPPORTED;
+  const WsLayout L = ws_layout(dtype, T, d_in, d_out, B, rp);
+  if (ws_bytes < L.total) return ISOPO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* w = (char*)ws;
+  int64_t* off_dev = (int64_t*)(w + L.off_offsets);
+  int32_t* tokseq = (int32_t*)(w + L.off_tokseq);
+  s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
+  if (s != ISOPO_OK) return s;
+  if (dtype == ISOPO_F32) {
+    if (rp == ISOPO_PATH_GRAM)
+      return f32_gram((const float*)X, (const float*)dY, T, d_in, d_out, tokseq, B, (double*)(w + L.off_kacc), K, st);
+    float* G = (float*)(w + L.off_G);
+    s = f32_seq_grad((const float*)X, (const float*)dY, d_in, d_out, off_dev, B, G, st);
+    if (s != ISOPO_OK) return s;
+    return f32_ntk(G, L.n_pad, B, K, st);
+  }
+  if (rp == ISOPO_PATH_GRAM) return bf16_gram(X, dY, T, d_in, d_out, tokseq, B, K, info, st);
+  void* G = w + L.off_G;
+  s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, B, L, G, info, st);
+  if (s != ISOPO_OK) return s;
+  return bf16_ntk(G, L, B, K, info, st);
+}
+
+isopo_status isopo_transform_advantages(const float* K, const float* A, int B, isopo_variant variant, float lambda,
+                                        const float* opt_pqr_regs, float* coeffs, int32_t* info, void* cuda_stream) {
+  if (!K || !A || !coeffs || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
+  if ((int)variant < 0 || (int)variant > (int)ISOPO_VAR_NORMALISED_RAW) return ISOPO_ERR_INVALID_ARG;
+  if (!(lambda >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
+  if (variant == ISOPO_VAR_GENERAL && !opt_pqr_regs) return ISOPO_ERR_INVALID_ARG;
+  if (variant == ISOPO_VAR_INTERACTING && B > 256) return ISOPO_ERR_UNSUPPORTED;
+  return transform(K, A, B, variant, lambda, opt_pqr_regs, coeffs, info, (cudaStream_t)cuda_stream);
+}
+
+isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                               const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
+                               float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  if (!coeffs || !dW || !info) return ISOPO_ERR_INVALID_ARG;
+  if (beta != 0.0f && beta != 1.0f) return ISOPO_ERR_INVALID_ARG;
+  isopo_status s = check_layer_args(X, dY, dtype, T, d_in, d_out, seq_offsets_host, B, path, ws);
+  if (s != ISOPO_OK) return s;
+  const isopo_path rp = resolve_path(dtype, T, d_in, d_out, B, path);
+  if (dtype == ISOPO_BF16 && rp == ISOPO_PATH_MATERIALISE && B > 256) return ISOPO_ERR_UNSUPPORTED;
+  const WsLayout L = ws_layout(dtype, T, d_in, d_out, B, rp);
+  if (ws_bytes < L.total) return ISOPO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* w = (char*)ws;
+  if (rp == ISOPO_PATH_MATERIALISE) {
+    if (dtype == ISOPO_F32) return f32_combine((const float*)(w + L.off_G), L.n_pad, B, coeffs, dW, beta, st);
+    return bf16_combine(w + L.off_G, L, d_in, d_out, B, coeffs, dW, beta, st);
+  }
+  // GEMM over all tokens: refresh the token -> sequence map so the call also works on its own.
+  int64_t* off_dev = (int64_t*)(w + L.off_offsets);
+  int32_t* tokseq = (int32_t*)(w + L.off_tokseq);
+  s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
+  if (s != ISOPO_OK) return s;
+  if (dtype == ISOPO_F32)
+    return f32_weight_grad((const float*)X, (const float*)dY, T, d_in, d_out, coeffs, tokseq, dW, beta, st);
+  return bf16_weight_grad(X, dY, T, d_in, d_out, coeffs, tokseq, dW, beta, info, st);
+}
+
+}  // extern "C"

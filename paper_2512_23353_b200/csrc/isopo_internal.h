@@ -1,0 +1,73 @@
+// Internal declarations shared by the translation units of libisopo (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "isopo.h"
+
+namespace isopo {
+
+// Tile of the stored per-sequence gradients on the bf16 path: one tensor-core accumulator tile.
+constexpr int kTileM = 128;  // rows of G (d_out)
+constexpr int kTileN = 256;  // columns of G (d_in)
+constexpr int kTileElems = kTileM * kTileN;
+
+// Identifiers written to *info together with ISOPO_INFO_TIMEOUT.
+enum KernelId : int { kIdSeqGrad = 1, kIdNtk = 2, kIdGram = 3, kIdWeightGrad = 4 };
+
+struct WsLayout {
+  size_t off_offsets;  // int64 [B+1]
+  size_t off_tokseq;   // int32 [T]
+  size_t off_kacc;     // float64 [B*B]   (float32 path: K accumulators)
+  size_t off_G;        // stored gradients (materialised path only)
+  size_t total;
+  int tiles_m, tiles_n;  // bf16 materialised layout: tiles per gradient
+  int64_t n_pad;         // elements per stored gradient (row stride of G_flat)
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path resolved);
+
+void set_cuda_error(cudaError_t e, const char* where);
+#define ISOPO_CUDA_TRY(expr)                                  \
+  do {                                                        \
+    cudaError_t e__ = (expr);                                 \
+    if (e__ != cudaSuccess) {                                 \
+      ::isopo::set_cuda_error(e__, #expr);                    \
+      return ISOPO_ERR_CUDA;                                  \
+    }                                                         \
+  } while (0)
+
+// ---- launchers (each enqueues on `st` and returns a status; none synchronises) ----
+
+isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq, cudaStream_t st);
+
+// float32 SIMT path
+isopo_status f32_seq_grad(const float* X, const float* dY, int d_in, int d_out, const int64_t* off_dev, int B,
+                          float* G, cudaStream_t st);
+isopo_status f32_ntk(const float* G, int64_t N, int B, float* K, cudaStream_t st);
+isopo_status f32_gram(const float* X, const float* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
+                      double* kacc, float* K, cudaStream_t st);
+isopo_status f32_combine(const float* G, int64_t N, int B, const float* coeffs, float* dW, float beta, cudaStream_t st);
+isopo_status f32_weight_grad(const float* X, const float* dY, int64_t T, int d_in, int d_out, const float* coeffs,
+                             const int32_t* tokseq, float* dW, float beta, cudaStream_t st);
+
+// bf16 tcgen05 path
+isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
+                           const int64_t* off_dev, int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st);
+isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t* info, cudaStream_t st);
+isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
+                          float beta, cudaStream_t st);
+isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
+                       float* K, int32_t* info, cudaStream_t st);
+isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* coeffs,
+                              const int32_t* tokseq, float* dW, float beta, int32_t* info, cudaStream_t st);
+
+// transform (all variants)
+isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* pqr_regs_host,
+                       float* coeffs, int32_t* info, cudaStream_t st);
+
+}  // namespace isopo

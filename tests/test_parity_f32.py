@@ -1,0 +1,111 @@
+"""GPU parity, float32 path: the library (through the C ABI) against the fp64 oracle, element by
+element on seeded inputs.  Tolerance: relative Frobenius error <= 1e-5 on K, coefficients and dW."""
+
+import numpy as np
+import pytest
+import torch
+
+from tests._util import offdiag_rel_fro, oracle_layer, rel_fro
+from paper_2512_23353_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2512_23353_b200 import binding
+    return binding
+
+
+def _run(b, X, dY, off, A, variant, lam, path, pqr_regs=None):
+    Xd, dYd, Ad = (torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in (X, dY, A))
+    res = b.isopo_layer(Xd, dYd, off, Ad, variant, lam, path, pqr_regs)
+    torch.cuda.synchronize()
+    K_o, c_o, dW_o = oracle_layer(Xd, dYd, off, Ad, variant, lam, pqr_regs)
+    return res, K_o, c_o, dW_o
+
+
+def _tiny(correlated=False):
+    w = wl.WORKLOADS["tiny_f32"]
+    off, A = wl.microbatch(w)
+    X, dY = wl.layer_inputs_host(w, w.layers[0], int(off[-1]), correlated)
+    return X, dY, off, A
+
+
+@pytest.mark.parametrize("path", ["gram", "materialise", "auto"])
+@pytest.mark.parametrize("correlated", [False, True])
+def test_tiny_config_all_variants(b, path, correlated):
+    X, dY, off, A = _tiny(correlated)
+    pcode = {"gram": b.PATH_GRAM, "materialise": b.PATH_MATERIALISE, "auto": b.PATH_AUTO}[path]
+    K_ref = oracle_layer(torch.from_numpy(X), torch.from_numpy(dY), off, torch.from_numpy(A), b.VAR_REINFORCE, 0.0)[0]
+    lam = 1e-3 * float(np.mean(np.diag(K_ref)))
+    cases = [(b.VAR_REINFORCE, 0.0, None), (b.VAR_NORMALISED, lam, None), (b.VAR_NORMALISED, 0.0, None),
+             (b.VAR_NORMALISED_RAW, lam, None), (b.VAR_DIRECTION, 1e-3, None), (b.VAR_EUCLID, lam, None),
+             (b.VAR_INTERACTING, lam, None),
+             (b.VAR_GENERAL, 0.0, [0.0, -1.0, -2.0, 0.0, 0.0, 0.0]),
+             (b.VAR_GENERAL, 0.0, [-0.5, 0.25, -1.0, 0.1 * lam, lam, 0.01])]
+    for variant, lm, g in cases:
+        res, K_o, c_o, dW_o = _run(b, X, dY, off, A, variant, lm, pcode, g)
+        assert res.info == 0
+        K = res.K.cpu().numpy()
+        assert np.array_equal(K, K.T)
+        assert rel_fro(K, K_o) <= TOL, (variant, rel_fro(K, K_o))
+        if correlated:
+            assert offdiag_rel_fro(K, K_o) <= TOL
+        nz = np.abs(c_o) > 0
+        assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL, (variant, rel_fro(res.coeffs.cpu().numpy(), c_o))
+        assert np.all(res.coeffs.cpu().numpy()[~nz] == 0)
+        assert rel_fro(res.dW.cpu().numpy(), dW_o) <= TOL, (variant, rel_fro(res.dW.cpu().numpy(), dW_o))
+
+
+@pytest.mark.parametrize("path", ["gram", "materialise"])
+@pytest.mark.parametrize("shape", [(1, 37, 24, 40), (13, 1, 40, 24), (5, 50, 72, 8), (3, 200, 100, 132)])
+def test_edge_shapes(b, path, shape):
+    """One sequence; every sequence a single token (K = (dY dY^T) o (X X^T)); widths that are not
+    tile multiples; lengths that straddle several staging chunks."""
+    B, Lmax, d_in, d_out = shape
+    rng = np.random.default_rng(B * 1000 + Lmax)
+    L = np.full(B, Lmax) if Lmax == 1 or B == 1 else rng.integers(1, Lmax + 1, size=B)
+    off = np.concatenate([[0], np.cumsum(L)]).astype(np.int64)
+    T = int(off[-1])
+    X = rng.standard_normal((T, d_in), dtype=np.float32)
+    dY = rng.standard_normal((T, d_out), dtype=np.float32)
+    A = rng.standard_normal(B).astype(np.float32)
+    pcode = b.PATH_GRAM if path == "gram" else b.PATH_MATERIALISE
+    for variant, lam in ((b.VAR_NORMALISED, 0.0), (b.VAR_INTERACTING, 0.5)):
+        res, K_o, c_o, dW_o = _run(b, X, dY, off, A, variant, lam, pcode)
+        assert res.info == 0
+        assert rel_fro(res.K.cpu().numpy(), K_o) <= TOL
+        assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL * max(1.0, np.linalg.cond(K_o + lam * np.eye(B)) / 100)
+        assert rel_fro(res.dW.cpu().numpy(), dW_o) <= TOL * max(1.0, np.linalg.cond(K_o + lam * np.eye(B)) / 100)
+    if Lmax == 1:
+        Kh = (dY.astype(np.float64) @ dY.astype(np.float64).T) * (X.astype(np.float64) @ X.astype(np.float64).T)
+        assert rel_fro(res.K.cpu().numpy(), Kh) <= TOL
+
+
+def test_beta_accumulates(b):
+    X, dY, off, A = _tiny()
+    Xd, dYd, Ad = (torch.from_numpy(a).cuda() for a in (X, dY, A))
+    for path in (b.PATH_GRAM, b.PATH_MATERIALISE):
+        res = b.isopo_layer(Xd, dYd, off, Ad, b.VAR_NORMALISED, 0.0, path)
+        ws = b.alloc_workspace(b.F32, X.shape[0], X.shape[1], dY.shape[1], len(off) - 1, path)
+        info = torch.zeros(1, dtype=torch.int32, device="cuda")
+        K = torch.empty_like(res.K)
+        b.isopo_layer_gram(Xd, dYd, off, K, ws, info, path)
+        base = torch.full_like(res.dW, 3.0)
+        b.isopo_weight_grad(Xd, dYd, res.coeffs, off, base, ws, info, path, beta=1.0)
+        torch.cuda.synchronize()
+        assert rel_fro((base - 3.0).cpu().numpy(), res.dW.cpu().numpy()) <= 1e-5
+
+
+def test_not_positive_definite_is_reported(b):
+    """An indefinite matrix (it cannot be a Gram matrix; lambda = 0) makes the second pivot
+    negative: the interacting transform must report its index instead of returning numbers."""
+    K = torch.tensor([[1.0, 2.0, 0.0], [2.0, 1.0, 0.0], [0.0, 0.0, 1.0]], device="cuda")
+    A = torch.tensor([1.0, -1.0, 0.5], device="cuda")
+    c = torch.empty(3, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.isopo_transform_advantages(K, A, b.VAR_INTERACTING, 0.0, c, info)
+    torch.cuda.synchronize()
+    assert int(info.item()) == 2
