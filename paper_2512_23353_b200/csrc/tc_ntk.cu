@@ -1,0 +1,248 @@
+// K = G_flat G_flat^T from the stored per-sequence gradients (Alg. 2 "make neural tangent kernel":
+// K_ij = sum(G_i * G_j)), and dW = sum_i c_i G_i from the same store (Alg. 2 last line).
+//
+// k_bf16_ntk: the B <= 256 stored gradients are the rows of a [B, n_pad] bf16 matrix.  Each CTA takes a
+// contiguous slab of the long contraction dimension, streams [B rows] x [64 elements] boxes through
+// a TMA ring, and uses every box as BOTH tcgen05 operands (K-major): rows 0..127 against all rows,
+// then rows 128..255 against rows 128..255 (the lower-left block is the mirror of the upper-right).
+// The float32 accumulators stay in tensor memory for the whole slab and are added into K once, with
+// reductions across CTAs by float atomics; a last tiny kernel mirrors the upper triangle.
+//
+// k_bf16_combine: pure streaming, one 16-byte chunk of every G_i per thread.
+#include "tc_common.cuh"
+
+namespace isopo {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kKB = 64;               // contraction elements per stage (one 128-byte row)
+constexpr int kStages = 6;
+constexpr int kStageBytes = 256 * 128;  // 256 rows x 128 bytes
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+
+struct NtkParams {
+  float* K;
+  int B;
+  long long nkb;  // 64-element blocks in the contraction dimension
+  int32_t* info;
+};
+
+__global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant__ CUtensorMap mapG, NtkParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  const uint32_t accfull_bar = bar0 + 8u * (2 * kStages);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(accfull_bar, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // this CTA's slab of the contraction dimension
+  const long long per = (p.nkb + gridDim.x - 1) / gridDim.x;
+  const long long kb0 = (long long)blockIdx.x * per, kb1 = min(p.nkb, kb0 + per);
+  const bool two = p.B > 128;                       // second row block present
+  const int rows = two ? 256 : 128;                 // rows per box (rows >= B arrive as zeros)
+  const uint32_t stage_tx = (uint32_t)rows * 128u;
+  const int n1 = two ? 256 : max(16, (p.B + 15) & ~15);
+  const int n2 = two ? max(16, (p.B - 128 + 15) & ~15) : 0;
+
+  if (kb0 < kb1) {
+    if (warp == 0) {
+      if (lane == 0) {
+        prefetch_tensormap(&mapG);
+        int stage = 0;
+        uint32_t phase = 0;
+        for (long long kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdNtk)) break;
+          mbar_arrive_expect_tx(full_bar(stage), stage_tx);
+          tma_load_2d(smem_base + stage * kStageBytes, &mapG, (int)(kb * kKB), 0, full_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    } else if (warp == 1) {
+      if (lane == 0) {
+        const uint32_t idesc1 = make_idesc_bf16(128, n1, false, false);
+        const uint32_t idesc2 = make_idesc_bf16(128, two ? n2 : 16, false, false);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (long long kb = kb0; kb < kb1; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.info, kIdNtk))) break;
+          tc_fence_after_sync();
+          const uint32_t base = smem_base + stage * kStageBytes;
+#pragma unroll
+          for (int k16 = 0; k16 < kKB / 16; ++k16) {
+            const bool accum = (kb > kb0) || k16 > 0;
+            const uint64_t d0 = make_sdesc_sw128(base + k16 * 32, 16, 1024);
+            mma_bf16(tmem_base, d0, d0, idesc1, accum);
+            if (two) {
+              const uint64_t d1 = make_sdesc_sw128(base + 128 * 128 + k16 * 32, 16, 1024);
+              mma_bf16(tmem_base + 256, d1, d1, idesc2, accum);
+            }
+          }
+          mma_commit(empty_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) mma_commit(accfull_bar);
+      }
+    } else {
+      const int q = warp & 3;
+      const int r = q * 32 + lane;
+      if (mbar_wait(accfull_bar, 0, abort_flag, p.info, kIdNtk)) {
+        tc_fence_after_sync();
+        const uint32_t tlane = (uint32_t)(q * 32) << 16;
+        // block A: rows 0..127 x columns 0..n1-1 of K; keep the upper triangle c >= r
+        for (int c0 = 0; c0 < n1; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + tlane + c0, v);
+          tmem_ld_wait();
+          if (r < p.B) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int c = c0 + e;
+              if (c >= r && c < p.B) atomicAdd(&p.K[(size_t)r * p.B + c], __uint_as_float(v[e]));
+            }
+          }
+        }
+        // block B: rows 128..255 x columns 128..255
+        if (two) {
+          const int rr = 128 + r;
+          for (int c0 = 0; c0 < n2; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_base + tlane + 256 + c0, v);
+            tmem_ld_wait();
+            if (rr < p.B) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                const int c = 128 + c0 + e;
+                if (c >= rr && c < p.B) atomicAdd(&p.K[(size_t)rr * p.B + c], __uint_as_float(v[e]));
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  if (*abort_flag) __nanosleep(100000);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+__global__ void k_mirror_upper(float* __restrict__ K, int B) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= B * B) return;
+  const int i = e / B, j = e % B;
+  if (j < i) K[e] = K[(size_t)j * B + i];
+}
+
+// dW = beta dW + sum_i c_i G_i.  One thread per 16-byte chunk position of the tile-blocked store.
+__global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long chunks /* n_pad / 8 */,
+                                                       int B, int tiles_n, int d_in, int d_out,
+                                                       const float* __restrict__ coeffs, float* __restrict__ dW,
+                                                       float beta) {
+  __shared__ float sc[256];
+  for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = coeffs[i];
+  __syncthreads();
+  for (long long pos = blockIdx.x * (long long)blockDim.x + threadIdx.x; pos < chunks;
+       pos += (long long)gridDim.x * blockDim.x) {
+    const int tile = (int)(pos / (kTileElems / 8)), rem = (int)(pos % (kTileElems / 8));
+    const int j = rem / kTileM, r = rem % kTileM;
+    const int m = (tile / tiles_n) * kTileM + r, n = (tile % tiles_n) * kTileN + j * 8;
+    if (m >= d_out || n >= d_in) continue;
+    float acc[8] = {};
+    const uint4* src = G + pos;
+    int i = 0;
+    for (; i + 8 <= B; i += 8) {
+      uint4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(i + u) * chunks);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float c = sc[i + u];
+        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
+          acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
+        }
+      }
+    }
+    for (; i < B; ++i) {
+      const uint4 v = __ldcs(src + (size_t)i * chunks);
+      const float c = sc[i];
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
+        acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
+      }
+    }
+    float4* out = reinterpret_cast<float4*>(dW + (size_t)m * d_in + n);
+    float4 o0 = make_float4(acc[0], acc[1], acc[2], acc[3]), o1 = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    if (beta != 0.f) {
+      const float4 p0 = out[0], p1 = out[1];
+      o0.x += p0.x; o0.y += p0.y; o0.z += p0.z; o0.w += p0.w;
+      o1.x += p1.x; o1.y += p1.y; o1.z += p1.z; o1.w += p1.w;
+    }
+    out[0] = o0;
+    out[1] = o1;
+  }
+}
+
+}  // namespace
+
+isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t* info, cudaStream_t st) {
+  if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  CUtensorMap mapG;
+  const uint32_t rows = B > 128 ? 256 : 128;
+  isopo_status s = make_map_2d_bf16(&mapG, G, (uint64_t)B, (uint64_t)L.n_pad, (uint64_t)L.n_pad, 64, rows);
+  if (s != ISOPO_OK) return s;
+  int dev = 0, sms = 0;
+  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
+  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_ntk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
+  NtkParams p{K, B, L.n_pad / kKB, info};
+  const int grid = (int)std::max<long long>(1, std::min<long long>(sms, p.nkb / 8));
+  k_bf16_ntk<<<grid, kThreads, kSmemBytes, st>>>(mapG, p);
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  k_mirror_upper<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
+                          float beta, cudaStream_t st) {
+  if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  const long long chunks = L.n_pad / 8;
+  int dev = 0, sms = 0;
+  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
+  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int grid = (int)std::min<long long>((chunks + 255) / 256, (long long)sms * 8);
+  k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta);
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+}  // namespace isopo
