@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the ISOPO per-layer hot path on B200.
+
+One "step" = the whole hot path (isopo_layer_gram -> isopo_transform_advantages -> isopo_weight_grad)
+for the seven projections of one transformer block over one ragged synthetic microbatch.  The
+default workload is the 1.5B-class block (d_model 1536, FFN 8960, kv 256; 256 sequences with
+log-uniform lengths in [256, 4096], ~355k tokens), the shapes the throughput target is quoted on.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own microbatch with no
+data-path collective (the path shards by independent microbatches) and the time is the max over
+ranks.  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "isopo_block_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ------------------------------------------------------------------------------------------------
+# helpers
+# ------------------------------------------------------------------------------------------------
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample(workload_name: str, n_seq: int, len_div: int):
+    """Bounded sample of the workload for the CPU oracle: the first `n_seq` sequences with every
+    length divided by `len_div`, all seven projections.  Returns (tokens, seconds, description)."""
+    from oracle import isopo_oracle as orc
+    from paper_2512_23353_b200 import workloads as wl
+
+    w = wl.WORKLOADS[workload_name]
+    off_full, A_full = wl.microbatch(w, scale_div=len_div)
+    off = off_full[: n_seq + 1].copy()
+    A = A_full[:n_seq].astype(np.float64)
+    T = int(off[-1])
+    inputs = []
+    for layer in w.layers:
+        X, dY = wl.layer_inputs_host(w, layer, T)
+        inputs.append((X, dY))
+    t0 = time.perf_counter()
+    for X, dY in inputs:
+        G = orc.sequence_gradients(X, dY, off)
+        K = orc.ntk(G)
+        lam = 1e-3 * float(np.mean(np.diag(K)))
+        c = orc.transform_advantages(K, A, orc.INTERACTING, lam)
+        orc.weight_gradient(G, c)
+    dt = time.perf_counter() - t0
+    desc = (f"{workload_name}: first {n_seq} of {w.B} sequences, lengths/{len_div} ({T} tokens), all "
+            f"{len(w.layers)} projections, interacting variant, numpy float64")
+    return T, dt, desc
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    times, tokens, desc = [], 0, ""
+    for it in range(args.warmup + args.steps):
+        tokens, dt, desc = oracle_sample(args.workload, args.cpu_seqs, args.cpu_len_div)
+        if it >= args.warmup:
+            times.append(dt)
+    ms = 1000.0 * sum(times) / len(times)
+    value = tokens / (ms / 1000.0)
+    cores = cpu_threads()
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+def run_gpu(args):
+    import torch
+
+    from paper_2512_23353_b200 import binding as b
+    from paper_2512_23353_b200 import workloads as wl
+
+    rank, world, local = dist_env()
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("launch with torchrun for --gpus > 1")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = wl.WORKLOADS[args.workload]
+    if world > 1:  # every rank its own microbatch
+        from dataclasses import replace
+        w = replace(w, seed=w.seed + 7919 * rank)
+    off, A_host = wl.microbatch(w)
+    T, B = int(off[-1]), w.B
+    dt_code = b.BF16 if w.dtype == "bf16" else b.F32
+    variant = b.VAR_INTERACTING if args.variant == "interacting" else b.VAR_NORMALISED
+
+    layers = []
+    ws_bytes = 0
+    for layer in w.layers:
+        X, dY = wl.layer_inputs_device(w, layer, T, dev)
+        path = b.isopo_choose_path(dt_code, T, layer.d_in, layer.d_out, B)
+        ws_bytes = max(ws_bytes, b.isopo_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, path))
+        layers.append({"layer": layer, "X": X, "dY": dY, "path": path,
+                       "K": torch.empty((B, B), dtype=torch.float32, device=dev),
+                       "c": torch.empty(B, dtype=torch.float32, device=dev),
+                       "dW": torch.zeros((layer.d_out, layer.d_in), dtype=torch.float32, device=dev),
+                       "lam": 0.0})
+    raw = torch.empty(ws_bytes + 1024, dtype=torch.uint8, device=dev)
+    shift = (-raw.data_ptr()) % 1024
+    ws = raw[shift:shift + ws_bytes]
+    A = torch.from_numpy(A_host).to(dev)
+    info = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        for L in layers:
+            b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
+            b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
+            b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+
+    # the regulariser is an absolute number the caller carries from earlier minibatches:
+    # 1e-3 * mean(diag K), taken once from an untimed pass
+    step()
+    torch.cuda.synchronize()
+    for L in layers:
+        L["lam"] = 1e-3 * float(torch.diagonal(L["K"]).mean().item())
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if int(info.item()) != 0:
+        raise SystemExit(f"device-side error during warm-up: info={int(info.item()):#x}")
+    b.isopo_profile_collect()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    b.isopo_profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    b.isopo_profile_enable(False)
+    elapsed_ms = e0.elapsed_time(e1)
+    prof = b.isopo_profile_collect()
+    if int(info.item()) != 0:
+        raise SystemExit(f"device-side error during the timed region: info={int(info.item()):#x}")
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+        tok = torch.tensor([T], dtype=torch.float64, device=dev)
+        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
+        total_tokens = float(tok.item())
+    else:
+        total_tokens = float(T)
+    ms_per_step = elapsed_ms / args.steps
+    value = total_tokens / (ms_per_step / 1000.0)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    # ---- algorithmic work of one step (this rank) ----
+    flops_dw = sum(2.0 * T * L["layer"].d_in * L["layer"].d_out for L in layers)
+    flops_k = sum(float(B) * B * L["layer"].d_in * L["layer"].d_out for L in layers)
+    flops_comb = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers)
+    flops_step = flops_dw + flops_k + flops_comb
+    step_tflops = flops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel, from the events recorded inside the timed region ----
+    dom = max(prof.items(), key=lambda kv: kv[1][0])[0] if prof else None
+    roofline = None
+    if dom == "k_bf16_seq_grad":
+        ms_total, n = prof[dom]
+        achieved = flops_dw * args.steps / (ms_total * 1e-3) / 1e12
+        roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
+                    "avg_launch_ms": ms_total / n, "launches": n}
+    elif dom is not None:
+        ms_total, n = prof[dom]
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": None, "traffic": None, "avg_launch_ms": ms_total / n, "launches": n}
+    kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items()}
+    g_bytes = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers)  # one pass over the stored gradients
+    for name in ("k_bf16_ntk", "k_bf16_combine"):
+        if name in kernels and kernels[name]["ms_per_step"] > 0:
+            kernels[name]["hbm_gbs"] = g_bytes / (kernels[name]["ms_per_step"] * 1e-3) / 1e9
+            kernels[name]["hbm_frac"] = kernels[name]["hbm_gbs"] / peaks["hbm_gbs"]
+
+    # ---- plain dW GEMM (cuBLAS through torch) on the same inputs, same run ----
+    plain_ms = 0.0
+    for L in layers:
+        for _ in range(3):
+            torch.matmul(L["dY"].t(), L["X"])
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            torch.matmul(L["dY"].t(), L["X"])
+        c.record()
+        torch.cuda.synchronize()
+        plain_ms += a.elapsed_time(c) / args.steps
+    overhead = ms_per_step / plain_ms
+
+    # ---- end to end: host buffers, copies inside the timed region ----
+    e2e = None
+    if not args.skip_e2e:
+        shapes = {}
+        for L in layers:
+            shapes.setdefault(("X", L["layer"].d_in), L["X"])
+            shapes.setdefault(("dY", L["layer"].d_out), L["dY"])
+        pinned = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in shapes.items()}
+        for k, v in shapes.items():
+            pinned[k].copy_(v)
+        dW_host = {id(L): torch.empty(L["dW"].shape, dtype=torch.float32, pin_memory=True) for L in layers}
+        h2d = sum(L["X"].numel() * L["X"].element_size() + L["dY"].numel() * L["dY"].element_size() for L in layers)
+        d2h = sum(L["dW"].numel() * 4 for L in layers)
+
+        def e2e_step():
+            for L in layers:
+                L["X"].copy_(pinned[("X", L["layer"].d_in)], non_blocking=True)
+                L["dY"].copy_(pinned[("dY", L["layer"].d_out)], non_blocking=True)
+                b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
+                b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
+                b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+                dW_host[id(L)].copy_(L["dW"], non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        n_e2e = max(1, min(args.steps, 3))
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        c.record()
+        torch.cuda.synchronize()
+        e2e_ms = a.elapsed_time(c) / n_e2e
+        e2e = {"value": T / (e2e_ms / 1000.0), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": n_e2e}
+        del pinned, dW_host
+
+    # ---- the oracle on this machine's host cores, bounded sample ----
+    cpu = None
+    if world == 1 and not args.skip_cpu:
+        tok_s, dt_s, desc = oracle_sample(args.workload, args.cpu_seqs, args.cpu_len_div)
+        cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
+               "seconds": dt_s}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": args.workload, "B": B, "tokens": T, "variant": args.variant,
+                   "layers": [f"{L['layer'].name}:{L['layer'].d_in}->{L['layer'].d_out}" for L in layers],
+                   "paths": ["gram" if L["path"] == b.PATH_GRAM else "materialise" for L in layers],
+                   "l2": "inputs larger than L2 (no flush needed)",
+                   "step": "layer_gram + transform_advantages + weight_grad for each projection"},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": int(sum(v[1] for v in prof.values())),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "step_tflops": step_tflops,
+        "pct_bf16_peak_sustained": step_tflops / peaks["bf16_tflops_sustained"],
+        "plain_dw_gemm_ms": plain_ms,
+        "overhead_vs_plain_dw_gemm": overhead,
+        "kernels": kernels,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llm_1p5b")
+    ap.add_argument("--variant", default="interacting", choices=["interacting", "normalised"])
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--cpu-seqs", type=int, default=8)
+    ap.add_argument("--cpu-len-div", type=int, default=8)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

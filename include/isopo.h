@@ -158,6 +158,18 @@ ISOPO_API isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dt
                                const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream);
 
+/*
+ * Measurement hooks (the paper has no counterpart).  While enabled, every kernel the library
+ * launches is bracketed by CUDA events on its stream.  isopo_profile_collect synchronises those
+ * events, adds the elapsed milliseconds and launch counts per kernel into the caller's arrays
+ * (host, ISOPO_NUM_KERNELS entries each, overwritten) and forgets them.  Launch counts are kept
+ * even while event timing is disabled.  Not thread-safe; meant for benchmarks.
+ */
+#define ISOPO_NUM_KERNELS 13
+ISOPO_API void isopo_profile_enable(int on);
+ISOPO_API isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_kernel);
+ISOPO_API const char* isopo_kernel_name(int kernel_id);
+
 #ifdef __cplusplus
 }
 #endif

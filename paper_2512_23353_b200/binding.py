@@ -26,7 +26,9 @@ INFO_TIMEOUT = 0x40000000
 EXPORTS = (
     "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",
     "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad",
+    "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name",
 )
+NUM_KERNELS = 13
 
 
 class IsopoError(RuntimeError):
@@ -60,6 +62,12 @@ def _load():
     lib.isopo_weight_grad.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
                                       c.c_void_p, c.c_int, c.c_int, c.c_void_p, c.c_float, c.c_void_p, c.c_size_t,
                                       c.c_void_p, c.c_void_p]
+    lib.isopo_profile_enable.restype = None
+    lib.isopo_profile_enable.argtypes = [c.c_int]
+    lib.isopo_profile_collect.restype = c.c_int
+    lib.isopo_profile_collect.argtypes = [c.c_void_p, c.c_void_p]
+    lib.isopo_kernel_name.restype = c.c_char_p
+    lib.isopo_kernel_name.argtypes = [c.c_int]
     return lib
 
 
@@ -149,6 +157,18 @@ def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, s
                                coeffs.data_ptr(), off.ctypes.data, B, path, dW.data_ptr(), float(beta),
                                ws.data_ptr(), ws.numel(), info.data_ptr(), _stream())
     _check(st, "isopo_weight_grad")
+
+
+def isopo_profile_enable(on: bool) -> None:
+    lib.isopo_profile_enable(1 if on else 0)
+
+
+def isopo_profile_collect() -> dict:
+    """{kernel name: (total ms, launches)} since the last collect; synchronises the recorded events."""
+    ms = np.zeros(NUM_KERNELS, dtype=np.float64)
+    n = np.zeros(NUM_KERNELS, dtype=np.int64)
+    _check(lib.isopo_profile_collect(ms.ctypes.data, n.ctypes.data), "isopo_profile_collect")
+    return {lib.isopo_kernel_name(k).decode(): (float(ms[k]), int(n[k])) for k in range(NUM_KERNELS) if n[k] or ms[k]}
 
 
 @dataclass

@@ -3,6 +3,7 @@
 // on the data and no CPU fallback.
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "isopo_internal.h"
 
@@ -12,6 +13,38 @@ static thread_local char g_cuda_err[256] = "no error";
 
 void set_cuda_error(cudaError_t e, const char* where) {
   snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
+}
+
+// ---- measurement hooks ----
+struct ProfRecord { int id; cudaEvent_t a, b; };
+static bool g_prof_on = false;
+static std::vector<ProfRecord> g_prof;
+static std::vector<cudaEvent_t> g_event_pool;
+static int64_t g_launches[kIdCount] = {};
+
+static cudaEvent_t take_event() {
+  if (!g_event_pool.empty()) {
+    cudaEvent_t e = g_event_pool.back();
+    g_event_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+LaunchScope::LaunchScope(int id, cudaStream_t st) : slot_(-1), st_(st) {
+  ++g_launches[id];
+  if (!g_prof_on) return;
+  ProfRecord r{id, take_event(), take_event()};
+  if (!r.a || !r.b) return;
+  cudaEventRecord(r.a, st);
+  slot_ = (int)g_prof.size();
+  g_prof.push_back(r);
+}
+
+LaunchScope::~LaunchScope() {
+  if (slot_ >= 0) cudaEventRecord(g_prof[slot_].b, st_);
 }
 
 WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path resolved) {
@@ -81,6 +114,32 @@ const char* isopo_status_string(isopo_status s) {
 }
 
 const char* isopo_last_cuda_error(void) { return g_cuda_err; }
+
+void isopo_profile_enable(int on) { g_prof_on = on != 0; }
+
+isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_kernel) {
+  if (!ms_by_kernel || !launches_by_kernel) return ISOPO_ERR_INVALID_ARG;
+  for (int k = 0; k < kIdCount; ++k) { ms_by_kernel[k] = 0.0; launches_by_kernel[k] = g_launches[k]; g_launches[k] = 0; }
+  isopo_status rc = ISOPO_OK;
+  for (const ProfRecord& r : g_prof) {
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(r.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.a, r.b);
+    if (e != cudaSuccess) { set_cuda_error(e, "isopo_profile_collect"); rc = ISOPO_ERR_CUDA; }
+    ms_by_kernel[r.id] += ms;
+    g_event_pool.push_back(r.a);
+    g_event_pool.push_back(r.b);
+  }
+  g_prof.clear();
+  return rc;
+}
+
+const char* isopo_kernel_name(int id) {
+  static const char* names[kIdCount] = {"k_tokseq", "k_bf16_seq_grad", "k_bf16_ntk", "k_bf16_gram", "k_bf16_weight_grad",
+                                        "k_bf16_combine", "k_transform", "k_mirror_upper", "k_f32_seq_grad",
+                                        "k_f32_ntk", "k_f32_gram", "k_f32_weight_grad", "k_f32_combine"};
+  return id >= 0 && id < kIdCount ? names[id] : "unknown";
+}
 
 isopo_path isopo_choose_path(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B) {
   if (!sizes_ok(dtype, T, d_in, d_out, B)) return ISOPO_PATH_GRAM;

@@ -14,8 +14,36 @@ constexpr int kTileM = 128;  // rows of G (d_out)
 constexpr int kTileN = 256;  // columns of G (d_in)
 constexpr int kTileElems = kTileM * kTileN;
 
-// Identifiers written to *info together with ISOPO_INFO_TIMEOUT.
-enum KernelId : int { kIdSeqGrad = 1, kIdNtk = 2, kIdGram = 3, kIdWeightGrad = 4 };
+// Kernel identifiers: written to *info together with ISOPO_INFO_TIMEOUT, and the index of the
+// per-kernel timing slots of isopo_profile_collect.
+enum KernelId : int {
+  kIdPrep = 0,
+  kIdSeqGrad = 1,
+  kIdNtk = 2,
+  kIdGram = 3,
+  kIdWeightGrad = 4,
+  kIdCombine = 5,
+  kIdTransform = 6,
+  kIdMirror = 7,
+  kIdF32SeqGrad = 8,
+  kIdF32Ntk = 9,
+  kIdF32Gram = 10,
+  kIdF32WeightGrad = 11,
+  kIdF32Combine = 12,
+  kIdCount = 13
+};
+
+// Brackets one kernel launch with CUDA events while profiling is enabled (isopo_profile_enable);
+// otherwise only counts the launch.
+class LaunchScope {
+ public:
+  LaunchScope(int id, cudaStream_t st);
+  ~LaunchScope();
+
+ private:
+  int slot_;
+  cudaStream_t st_;
+};
 
 struct WsLayout {
   size_t off_offsets;  // int64 [B+1]

@@ -191,7 +191,10 @@ isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off
                          cudaStream_t st) {
   ISOPO_CUDA_TRY(cudaMemcpyAsync(off_dev, off_host, sizeof(int64_t) * (size_t)(B + 1), cudaMemcpyHostToDevice, st));
   const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
-  k_tokseq<<<grid, 256, 0, st>>>(off_dev, B, T, tokseq);
+  {
+    LaunchScope scope(kIdPrep, st);
+    k_tokseq<<<grid, 256, 0, st>>>(off_dev, B, T, tokseq);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
@@ -200,14 +203,20 @@ isopo_status f32_seq_grad(const float* X, const float* dY, int d_in, int d_out, 
                           float* G, cudaStream_t st) {
   dim3 grid((d_in + kT - 1) / kT, (d_out + kT - 1) / kT, B);
   if (grid.y > 65535 || grid.z > 65535) return ISOPO_ERR_UNSUPPORTED;
-  k_f32_seq_grad<<<grid, 256, 0, st>>>(X, dY, d_in, d_out, off_dev, G);
+  {
+    LaunchScope scope(kIdF32SeqGrad, st);
+    k_f32_seq_grad<<<grid, 256, 0, st>>>(X, dY, d_in, d_out, off_dev, G);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
 
 isopo_status f32_ntk(const float* G, int64_t N, int B, float* K, cudaStream_t st) {
   if (B > 65535) return ISOPO_ERR_UNSUPPORTED;
-  k_f32_ntk<<<dim3(B, B), 256, 0, st>>>(G, N, B, K);
+  {
+    LaunchScope scope(kIdF32Ntk, st);
+    k_f32_ntk<<<dim3(B, B), 256, 0, st>>>(G, N, B, K);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
@@ -217,9 +226,15 @@ isopo_status f32_gram(const float* X, const float* dY, int64_t T, int d_in, int 
   const int64_t nt = (T + kGT - 1) / kGT;
   if (nt > 65535) return ISOPO_ERR_UNSUPPORTED;
   ISOPO_CUDA_TRY(cudaMemsetAsync(kacc, 0, sizeof(double) * (size_t)B * B, st));
-  k_f32_gram<<<dim3((unsigned)nt, (unsigned)nt), 256, 0, st>>>(X, dY, T, d_in, d_out, tokseq, B, kacc);
+  {
+    LaunchScope scope(kIdF32Gram, st);
+    k_f32_gram<<<dim3((unsigned)nt, (unsigned)nt), 256, 0, st>>>(X, dY, T, d_in, d_out, tokseq, B, kacc);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
-  k_f32_gram_finish<<<(B * B + 255) / 256, 256, 0, st>>>(kacc, B, K);
+  {
+    LaunchScope scope(kIdMirror, st);
+    k_f32_gram_finish<<<(B * B + 255) / 256, 256, 0, st>>>(kacc, B, K);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
@@ -227,7 +242,10 @@ isopo_status f32_gram(const float* X, const float* dY, int64_t T, int d_in, int 
 isopo_status f32_combine(const float* G, int64_t N, int B, const float* coeffs, float* dW, float beta,
                          cudaStream_t st) {
   const int grid = (int)std::min<int64_t>((N + 255) / 256, 148 * 8);
-  k_f32_combine<<<grid, 256, 0, st>>>(G, N, B, coeffs, dW, beta);
+  {
+    LaunchScope scope(kIdF32Combine, st);
+    k_f32_combine<<<grid, 256, 0, st>>>(G, N, B, coeffs, dW, beta);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
@@ -241,7 +259,10 @@ isopo_status f32_weight_grad(const float* X, const float* dY, int64_t T, int d_i
   int64_t splits = std::max<int64_t>(1, std::min<int64_t>((T + 255) / 256, (148 * 4 + gx * gy - 1) / (gx * gy)));
   int64_t slab = ((T + splits - 1) / splits + kTK - 1) / kTK * kTK;
   splits = (T + slab - 1) / slab;
-  k_f32_weight_grad<<<dim3(gx, gy, (unsigned)splits), 256, 0, st>>>(X, dY, T, d_in, d_out, coeffs, tokseq, dW, slab);
+  {
+    LaunchScope scope(kIdF32WeightGrad, st);
+    k_f32_weight_grad<<<dim3(gx, gy, (unsigned)splits), 256, 0, st>>>(X, dY, T, d_in, d_out, coeffs, tokseq, dW, slab);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }

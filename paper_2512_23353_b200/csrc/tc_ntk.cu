@@ -225,9 +225,15 @@ isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t
   ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
   NtkParams p{K, B, L.n_pad / kKB, info};
   const int grid = (int)std::max<long long>(1, std::min<long long>(sms, p.nkb / 8));
-  k_bf16_ntk<<<grid, kThreads, kSmemBytes, st>>>(mapG, p);
+  {
+    LaunchScope scope(kIdNtk, st);
+    k_bf16_ntk<<<grid, kThreads, kSmemBytes, st>>>(mapG, p);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
-  k_mirror_upper<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
+  {
+    LaunchScope scope(kIdMirror, st);
+    k_mirror_upper<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
@@ -240,7 +246,10 @@ isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out,
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   const int grid = (int)std::min<long long>((chunks + 255) / 256, (long long)sms * 8);
-  k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta);
+  {
+    LaunchScope scope(kIdCombine, st);
+    k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }

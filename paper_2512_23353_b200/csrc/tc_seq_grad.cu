@@ -204,7 +204,10 @@ isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, i
   SeqGradParams p{off_dev, (__nv_bfloat16*)G, L.n_pad, B, L.tiles_m, L.tiles_n, info};
   const long long units = (long long)B * L.tiles_m * L.tiles_n;
   const int grid = (int)std::min<long long>(units, sms);
-  k_bf16_seq_grad<<<grid, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
+  {
+    LaunchScope scope(kIdSeqGrad, st);
+    k_bf16_seq_grad<<<grid, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }

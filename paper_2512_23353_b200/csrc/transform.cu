@@ -1,15 +1,16 @@
 // Advantage transform: one CTA turns (K, A) into the per-sequence coefficients.
 //   simple variants  - per-row sums of K in float64, one warp per row
-//   interacting      - Cholesky of the packed lower triangle of K + lambda*I in shared memory
-//                      (float32), triangular solves by one warp, two refinement rounds with
-//                      float64 residuals taken from the float32 K in global memory
+//   interacting      - blocked Cholesky of K + lambda*I in shared memory (float32, 32 x 32 blocks,
+//                      warp-level diagonal factorisation), blocked triangular solves, then up to
+//                      two refinement rounds with float64 residuals taken from the float32 K,
+//                      stopped once the relative residual is below 1e-7
 #include "isopo_internal.h"
 
 namespace isopo {
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kMaxB = 256;
 
 struct TransformParams {
@@ -23,40 +24,190 @@ struct TransformParams {
   float p, q, r, reg_F, reg_G, reg_rel;
 };
 
-__device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }  // i >= j
 
 __device__ __forceinline__ double warp_sum(double v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
 
-// Solves L L^T x = b for one right-hand side held in shared memory (overwritten by x); warp 0 only.
-// Each lane owns entries lane, lane+32, ...
-__device__ void warp_cholesky_solve(const float* __restrict__ Lp, float* __restrict__ v, int B) {
+// ---------------------------------------------------------------------------------------------
+// Interacting variant: blocked Cholesky in shared memory.
+//
+// K + lambda*I is held as 32 x 32 blocks (lower block triangle, block (I,J) at slot I(I+1)/2+J),
+// every block column-major: element (r, c) at [c*32 + r], so that a warp whose lane owns row r
+// reads a block column without bank conflicts and 4 consecutive rows form one float4.
+// Per block column J:  (1) warp 0 factors the diagonal block in registers (shuffles) and inverts
+// the triangular factor;  (2) one warp per block below applies the inverse (a triangular solve
+// without divisions);  (3) one warp per trailing block does the rank-32 update with 4 x 8
+// register tiles.  The solves use the stored inverses of the diagonal blocks.
+// ---------------------------------------------------------------------------------------------
+constexpr int kNB = 32;
+constexpr int kBlk = kNB * kNB;
+
+__device__ __forceinline__ int blk_slot(int I, int J) { return I * (I + 1) / 2 + J; }
+
+// Column sums over the warp: on entry lane l holds r[c] = M[l][c]; on return r[0] of lane c holds
+// sum_l M[l][c].  Recursive halving: 31 shuffles for all 32 sums.
+__device__ __forceinline__ float warp_column_sums(float (&r)[kNB]) {
   const int lane = threadIdx.x & 31;
-  // forward: L y = b, column sweep
-  for (int k = 0; k < B; ++k) {
-    __syncwarp();
-    const float yk = v[k] / Lp[tri(k, k)];
-    __syncwarp();
-    if (lane == (k & 31)) v[k] = yk;
-    for (int i = k + 1 + lane; i < B; i += 32) v[i] = fmaf(-Lp[tri(i, k)], yk, v[i]);
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int idx = 0; idx < o; ++idx) {
+      const float send = up ? r[idx] : r[idx + o];
+      const float keep = up ? r[idx + o] : r[idx];
+      r[idx] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+    }
   }
-  // backward: L^T x = y, row sweep
-  for (int k = B - 1; k >= 0; --k) {
-    __syncwarp();
-    const float xk = v[k] / Lp[tri(k, k)];
-    __syncwarp();
-    if (lane == (k & 31)) v[k] = xk;
-    for (int i = lane; i < k; i += 32) v[i] = fmaf(-Lp[tri(k, i)], xk, v[i]);
-  }
-  __syncwarp();
+  return r[0];
 }
+
+// Factors the 32 x 32 diagonal block D (column-major, symmetric input) in place into its lower
+// Cholesky factor and writes the inverse of that factor to Inv (column-major).  One warp.
+// Returns 0, or the 1-based local index of the first non-positive pivot.
+__device__ __noinline__ int warp_factor_diag(float* __restrict__ D, float* __restrict__ Inv) {
+  const int lane = threadIdx.x & 31;
+  float r[kNB];
+#pragma unroll
+  for (int c = 0; c < kNB; ++c) r[c] = D[c * kNB + lane];  // row `lane`
+  int fail = 0;
+  float rdiag = 0.f;  // 1 / L[lane][lane]
+#pragma unroll
+  for (int k = 0; k < kNB; ++k) {
+    const float d = __shfl_sync(0xffffffffu, r[k], k);
+    if (!(d > 0.f) && fail == 0) fail = k + 1;
+    const float rs = rsqrtf(d);
+    if (lane == k) rdiag = rs;
+    r[k] = lane == k ? d * rs : r[k] * rs;  // L[lane][k] (rows above k hold junk, never used)
+#pragma unroll
+    for (int j = k + 1; j < kNB; ++j) {
+      const float ljk = __shfl_sync(0xffffffffu, r[k], j);
+      r[j] = fmaf(-r[k], ljk, r[j]);
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < kNB; ++c) D[c * kNB + lane] = c <= lane ? r[c] : 0.f;
+  __syncwarp();
+  // inverse, column sweep: lane j solves L z = e_j; after step k, z[k] = Inv[k][j] is final
+  float z[kNB];
+#pragma unroll
+  for (int i = 0; i < kNB; ++i) z[i] = i == lane ? 1.f : 0.f;
+#pragma unroll
+  for (int k = 0; k < kNB; ++k) {
+    z[k] *= __shfl_sync(0xffffffffu, rdiag, k);
+#pragma unroll
+    for (int i = k + 1; i < kNB; ++i) z[i] = fmaf(-D[k * kNB + i], z[k], z[i]);  // L[i][k], broadcast
+  }
+#pragma unroll
+  for (int i = 0; i < kNB; ++i) Inv[lane * kNB + i] = z[i];
+  return fail;
+}
+
+// X = A * Inv^T for one 32 x 32 block A (in place); lane owns a row.  Inv lower triangular.
+__device__ __noinline__ void warp_apply_inverse(float* __restrict__ A, const float* __restrict__ Inv) {
+  const int lane = threadIdx.x & 31;
+  float a[kNB], x[kNB];
+#pragma unroll
+  for (int c = 0; c < kNB; ++c) { a[c] = A[c * kNB + lane]; x[c] = 0.f; }
+#pragma unroll
+  for (int p = 0; p < kNB; ++p)
+#pragma unroll
+    for (int k = p; k < kNB; ++k) x[k] = fmaf(a[p], Inv[p * kNB + k], x[k]);  // Inv[k][p], broadcast
+#pragma unroll
+  for (int c = 0; c < kNB; ++c) A[c * kNB + lane] = x[c];
+}
+
+// C -= A * Bm^T for 32 x 32 blocks (all column-major); lane computes a 4 x 8 sub-tile.
+__device__ __noinline__ void warp_rank32_update(float* __restrict__ C, const float* __restrict__ A,
+                                                const float* __restrict__ Bm) {
+  const int lane = threadIdx.x & 31, r0 = (lane & 7) * 4, c0 = (lane >> 3) * 8;
+  float4 acc[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) acc[c] = *reinterpret_cast<const float4*>(C + (c0 + c) * kNB + r0);
+#pragma unroll 8
+  for (int p = 0; p < kNB; ++p) {
+    const float4 a = *reinterpret_cast<const float4*>(A + p * kNB + r0);
+    const float4 b0 = *reinterpret_cast<const float4*>(Bm + p * kNB + c0);
+    const float4 b1 = *reinterpret_cast<const float4*>(Bm + p * kNB + c0 + 4);
+    const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      acc[c].x = fmaf(-a.x, b[c], acc[c].x);
+      acc[c].y = fmaf(-a.y, b[c], acc[c].y);
+      acc[c].z = fmaf(-a.z, b[c], acc[c].z);
+      acc[c].w = fmaf(-a.w, b[c], acc[c].w);
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < 8; ++c) *reinterpret_cast<float4*>(C + (c0 + c) * kNB + r0) = acc[c];
+}
+
+// Solves L L^T x = v in place (v in shared memory, nb*32 entries) with the blocked factor.
+__device__ __noinline__ void block_cholesky_solve(const float* __restrict__ Lb, const float* __restrict__ InvD,
+                                                  float* __restrict__ v, int nb) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  // forward: L y = v
+  for (int J = 0; J < nb; ++J) {
+    if (warp == 0) {
+      const float* Inv = InvD + J * kBlk;
+      float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < kNB; k += 2) {
+        acc0 = fmaf(Inv[k * kNB + lane], v[J * kNB + k], acc0);
+        acc1 = fmaf(Inv[(k + 1) * kNB + lane], v[J * kNB + k + 1], acc1);
+      }
+      __syncwarp();
+      v[J * kNB + lane] = acc0 + acc1;
+    }
+    __syncthreads();
+    for (int I = J + 1 + warp; I < nb; I += nwarps) {
+      const float* L = Lb + blk_slot(I, J) * kBlk;
+      float acc0 = v[I * kNB + lane], acc1 = 0.f;
+#pragma unroll
+      for (int p = 0; p < kNB; p += 2) {
+        acc0 = fmaf(-L[p * kNB + lane], v[J * kNB + p], acc0);
+        acc1 = fmaf(-L[(p + 1) * kNB + lane], v[J * kNB + p + 1], acc1);
+      }
+      v[I * kNB + lane] = acc0 + acc1;
+    }
+    __syncthreads();
+  }
+  // backward: L^T x = y; lane owns a row of the block, column sums by recursive halving
+  for (int J = nb - 1; J >= 0; --J) {
+    if (warp == 0) {
+      const float* Inv = InvD + J * kBlk;
+      const float yj = v[J * kNB + lane];
+      float r[kNB];
+#pragma unroll
+      for (int i = 0; i < kNB; ++i) r[i] = Inv[i * kNB + lane] * yj;  // Inv[lane][i] y_lane
+      v[J * kNB + lane] = warp_column_sums(r);                        // x_i = sum_k Inv[k][i] y_k
+    }
+    __syncthreads();
+    for (int I = warp; I < J; I += nwarps) {
+      const float* L = Lb + blk_slot(J, I) * kBlk;  // y_I -= L_JI^T x_J
+      const float xj = v[J * kNB + lane];
+      float r[kNB];
+#pragma unroll
+      for (int i = 0; i < kNB; ++i) r[i] = L[i * kNB + lane] * xj;
+      v[I * kNB + lane] -= warp_column_sums(r);
+    }
+    __syncthreads();
+  }
+}
+
+#ifdef ISOPO_PHASE_TIMERS
+__device__ long long g_phase[16];
+#define PHASE(n) do { if (threadIdx.x == 0) g_phase[n] = clock64(); } while (0)
+#define PHASE_ACC(n, t0) do { if (threadIdx.x == 0) { long long t1__ = clock64(); g_phase[n] += t1__ - t0; t0 = t1__; } } while (0)
+#else
+#define PHASE(n) do {} while (0)
+#define PHASE_ACC(n, t0) do {} while (0)
+#endif
 
 __global__ void __launch_bounds__(kThreads) k_transform(TransformParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ double s_trace;
-  __shared__ float s_pivot;
+  __shared__ double s_trace, s_res;
   __shared__ int s_fail;
   const int B = P.B, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kThreads / 32;
   const float* __restrict__ K = P.K;
@@ -108,57 +259,153 @@ __global__ void __launch_bounds__(kThreads) k_transform(TransformParams P) {
   }
 
   // ---------------- interacting: (K + lambda I) c = A ----------------
-  float* Lp = reinterpret_cast<float*>(smem_raw);                    // packed lower triangle
-  float* vec = Lp + (size_t)B * (B + 1) / 2;                          // right-hand side / correction
-  double* sol = reinterpret_cast<double*>(vec + ((B + 3) & ~3) + ((((size_t)B * (B + 1) / 2) & 1) ? 1 : 0));
+  const int nb = (B + kNB - 1) / kNB, Bp = nb * kNB;
+  float* Lb = reinterpret_cast<float*>(smem_raw);           // nb(nb+1)/2 blocks
+  float* InvD = Lb + (size_t)(nb * (nb + 1) / 2) * kBlk;    // nb inverse diagonal factors
+  float* vec = InvD + (size_t)nb * kBlk;                    // Bp floats
+  double* sol = reinterpret_cast<double*>(vec + Bp);        // Bp doubles (8-byte aligned: all counts even)
   if (tid == 0) s_fail = 0;
-  for (int e = tid; e < B * B; e += kThreads) {
-    const int i = e / B, j = e % B;
-    if (j <= i) Lp[tri(i, j)] = K[e] + (i == j ? P.lambda : 0.f);
+  PHASE(0);
+  // load the lower block triangle.  K is symmetric, so row j of K read along i gives column j of
+  // the blocks; float4 loads, eight in flight per thread, when B is a multiple of 4.
+  if ((B & 3) == 0) {
+    const int nvec = B * B / 4;
+    for (int base = tid; base < nvec; base += kThreads * 8) {
+      float4 val[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + u * kThreads;
+        val[u] = e < nvec ? __ldg(reinterpret_cast<const float4*>(K) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + u * kThreads;
+        if (e >= nvec) continue;
+        const int j = (e * 4) / B, i = (e * 4) % B, I = i / kNB, J = j / kNB;
+        if (I < J) continue;
+        float4 w = val[u];
+        if (i == j) w.x += P.lambda;
+        if (i + 1 == j) w.y += P.lambda;
+        if (i + 2 == j) w.z += P.lambda;
+        if (i + 3 == j) w.w += P.lambda;
+        *reinterpret_cast<float4*>(Lb + blk_slot(I, J) * kBlk + (j % kNB) * kNB + (i % kNB)) = w;
+      }
+    }
+  } else {
+    for (int e = tid; e < B * B; e += kThreads) {
+      const int j = e / B, i = e % B, I = i / kNB, J = j / kNB;
+      if (I >= J) Lb[blk_slot(I, J) * kBlk + (j % kNB) * kNB + (i % kNB)] = K[e] + (i == j ? P.lambda : 0.f);
+    }
+  }
+  // identity padding of the last block row / column
+  for (int e = tid; e < (Bp - B) * Bp; e += kThreads) {
+    const int i = B + e / Bp, j = e % Bp;  // rows B..Bp-1, all columns j <= i
+    if (j <= i || j / kNB == i / kNB)
+      Lb[blk_slot(i / kNB, j / kNB) * kBlk + (j % kNB) * kNB + (i % kNB)] = i == j ? 1.f : 0.f;
   }
   __syncthreads();
-  // left-looking Cholesky, thread i owns row i
-  for (int k = 0; k < B; ++k) {
-    float s = 0.f;
-    const int i = tid;
-    if (i >= k && i < B) {
-      const float* ri = Lp + tri(i, 0);
-      const float* rk = Lp + tri(k, 0);
-      s = ri[k];
-      for (int p = 0; p < k; ++p) s = fmaf(-ri[p], rk[p], s);
-      if (i == k) s_pivot = s;
+  PHASE(1);
+  long long tph = clock64();
+  (void)tph;
+  for (int J = 0; J < nb; ++J) {
+    if (warp == 0) {
+      const int f = warp_factor_diag(Lb + blk_slot(J, J) * kBlk, InvD + J * kBlk);
+      if (f != 0 && lane == 0) { s_fail = J * kNB + f; }
     }
     __syncthreads();
-    const float piv = s_pivot;
-    if (!(piv > 0.f)) {
-      if (tid == 0) { s_fail = 1; atomicCAS(P.info, 0, k + 1); }
-      break;
-    }
-    if (i >= k && i < B) Lp[tri(i, k)] = i == k ? sqrtf(piv) : s * rsqrtf(piv);
+    PHASE_ACC(8, tph);
+    if (s_fail) break;
+    for (int I = J + 1 + warp; I < nb; I += nwarps) warp_apply_inverse(Lb + blk_slot(I, J) * kBlk, InvD + J * kBlk);
     __syncthreads();
+    PHASE_ACC(9, tph);
+    // trailing blocks (I, Kc) with I >= Kc > J, one per warp
+    const int m = nb - 1 - J, ntrail = m * (m + 1) / 2;
+    for (int t = warp; t < ntrail; t += nwarps) {
+      int a = 0, rem = t;
+      while (rem > a) { rem -= a + 1; ++a; }  // t = a(a+1)/2 + rem, rem <= a
+      const int I = J + 1 + a, Kc = J + 1 + rem;
+      warp_rank32_update(Lb + blk_slot(I, Kc) * kBlk, Lb + blk_slot(I, J) * kBlk, Lb + blk_slot(Kc, J) * kBlk);
+    }
+    __syncthreads();
+    PHASE_ACC(10, tph);
   }
   __syncthreads();
   if (s_fail) {
+    if (tid == 0) atomicCAS(P.info, 0, s_fail);
     for (int i = tid; i < B; i += kThreads) P.coeffs[i] = 0.f;
     return;
   }
-  // initial solve + two refinement rounds
-  for (int i = tid; i < B; i += kThreads) { vec[i] = P.A[i]; sol[i] = 0.0; }
+  PHASE(2);
+  // solve, then refinement rounds with a float64 residual while it is above float32 round-off
+  double anorm2 = 0.0;
+  for (int i = tid; i < Bp; i += kThreads) {
+    const float a = i < B ? P.A[i] : 0.f;
+    vec[i] = a;
+    sol[i] = 0.0;
+    anorm2 += (double)a * a;
+  }
+  anorm2 = warp_sum(anorm2);
+  if (tid == 0) { s_trace = 0.0; s_res = 0.0; }
   __syncthreads();
+  if (lane == 0) atomicAdd(&s_trace, anorm2);
+  __syncthreads();
+  anorm2 = s_trace;
   for (int round = 0; round < 3; ++round) {
-    if (warp == 0) warp_cholesky_solve(Lp, vec, B);
-    __syncthreads();
-    for (int i = tid; i < B; i += kThreads) sol[i] += (double)vec[i];
+    block_cholesky_solve(Lb, InvD, vec, nb);
+    PHASE(3 + 2 * round);
+    for (int i = tid; i < Bp; i += kThreads) sol[i] += (double)vec[i];
     __syncthreads();
     if (round == 2) break;
-    // residual r = A - (K + lambda I) sol in float64
-    for (int i = warp; i < B; i += nwarps) {
-      double acc = 0.0;
-      for (int j = lane; j < B; j += 32) acc += (double)K[(size_t)i * B + j] * sol[j];
-      acc = warp_sum(acc);
-      if (lane == 0) vec[i] = (float)((double)P.A[i] - acc - (double)P.lambda * sol[i]);
+    double rn2 = 0.0;
+    for (int i0 = warp * 4; i0 < B; i0 += nwarps * 4) {  // four rows per warp pass: independent loads
+      double acc[4] = {0.0, 0.0, 0.0, 0.0};
+      if ((B & 3) == 0) {
+        for (int j0 = lane * 4; j0 < B; j0 += 256) {  // two float4 per lane and row in flight
+          float4 kv[4][2];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int j = j0 + h * 128;
+              kv[u][h] = (i0 + u < B && j < B) ? __ldg(reinterpret_cast<const float4*>(K + (size_t)(i0 + u) * B + j))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int j = j0 + h * 128;
+            if (j >= B) continue;
+            const double s0 = sol[j], s1 = sol[j + 1], s2 = sol[j + 2], s3 = sol[j + 3];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              acc[u] += (double)kv[u][h].x * s0 + (double)kv[u][h].y * s1 + (double)kv[u][h].z * s2 +
+                        (double)kv[u][h].w * s3;
+          }
+        }
+      } else {
+        for (int j = lane; j < B; j += 32) {
+          const double sj = sol[j];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (i0 + u < B) acc[u] += (double)K[(size_t)(i0 + u) * B + j] * sj;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const double a = warp_sum(acc[u]);
+        if (lane == 0 && i0 + u < B) {
+          const double r = (double)P.A[i0 + u] - a - (double)P.lambda * sol[i0 + u];
+          vec[i0 + u] = (float)r;
+          rn2 += r * r;
+        }
+      }
     }
+    if (lane == 0) atomicAdd(&s_res, rn2);
     __syncthreads();
+    PHASE(4);
+    const bool done = s_res <= 1e-14 * anorm2;  // relative residual below 1e-7
+    __syncthreads();
+    if (tid == 0) s_res = 0.0;
+    if (done) break;
   }
   for (int i = tid; i < B; i += kThreads) P.coeffs[i] = (float)sol[i];
 }
@@ -173,14 +420,14 @@ isopo_status transform(const float* K, const float* A, int B, isopo_variant v, f
   size_t smem = 0;
   if (v == ISOPO_VAR_INTERACTING) {
     if (B > kMaxB) return ISOPO_ERR_UNSUPPORTED;
-    smem = sizeof(float) * ((size_t)B * (B + 1) / 2 + (size_t)B + 8) + sizeof(double) * (size_t)B + 16;
-    static bool attr_set = false;  // idempotent; a race only repeats the same call
-    if (!attr_set) {
-      ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_transform, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-      attr_set = true;
-    }
+    const size_t nb = (size_t)(B + kNB - 1) / kNB;
+    smem = sizeof(float) * ((nb * (nb + 1) / 2 + nb) * kBlk + nb * kNB) + sizeof(double) * nb * kNB;
+    ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_transform, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   }
-  k_transform<<<1, kThreads, smem, st>>>(P);
+  {
+    LaunchScope scope(kIdTransform, st);
+    k_transform<<<1, kThreads, smem, st>>>(P);
+  }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }

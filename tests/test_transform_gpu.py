@@ -1,0 +1,74 @@
+"""GPU parity of isopo_transform_advantages alone: random Gram matrices of every block shape the
+blocked Cholesky meets (B below, at and above multiples of 32, up to the 256 limit)."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import isopo_oracle as orc
+from tests._util import VARIANT_NAME, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2512_23353_b200 import binding
+    return binding
+
+
+def _gram(B, rank_extra, seed):
+    """K = J J^T in float32 with strongly overlapping rows (a shared low-rank part)."""
+    rng = np.random.default_rng(seed)
+    J = rng.standard_normal((B, 4 * B + 8)) + 2.0 * rng.standard_normal((B, rank_extra)) @ rng.standard_normal((rank_extra, 4 * B + 8))
+    K = (J @ J.T).astype(np.float32)
+    return np.ascontiguousarray((K + K.T) / 2)
+
+
+@pytest.mark.parametrize("B", [1, 2, 31, 32, 33, 64, 100, 200, 255, 256])
+def test_interacting_solve(b, B):
+    K = _gram(B, 3, B)
+    A = np.random.default_rng(B + 1).standard_normal(B).astype(np.float32)
+    for rel in (1e-3, 1.0):
+        lam = np.float32(rel * np.mean(np.diag(K)))
+        Kd, Ad = torch.from_numpy(K).cuda(), torch.from_numpy(A).cuda()
+        c = torch.empty(B, device="cuda")
+        info = torch.zeros(1, dtype=torch.int32, device="cuda")
+        b.isopo_transform_advantages(Kd, Ad, b.VAR_INTERACTING, float(lam), c, info)
+        torch.cuda.synchronize()
+        assert int(info.item()) == 0
+        want = orc.transform_advantages(K.astype(np.float64), A.astype(np.float64), orc.INTERACTING, float(lam))
+        cond = np.linalg.cond(K.astype(np.float64) + float(lam) * np.eye(B))
+        # float32 storage of c (6e-8) plus a refined float32 factorisation: far below 1e-5 for these conditions
+        assert rel_fro(c.cpu().numpy(), want) <= max(1e-6, 1e-9 * cond), (B, rel, cond, rel_fro(c.cpu().numpy(), want))
+
+
+@pytest.mark.parametrize("B", [5, 64, 256, 300, 1000])
+def test_simple_variants_any_B(b, B):
+    K = _gram(B, 2, 7 * B)
+    A = np.random.default_rng(B).standard_normal(B).astype(np.float32)
+    Kd, Ad = torch.from_numpy(K).cuda(), torch.from_numpy(A).cuda()
+    lam = float(np.float32(0.01 * np.mean(np.diag(K))))
+    for variant, g in ((b.VAR_NORMALISED, None), (b.VAR_NORMALISED_RAW, None), (b.VAR_DIRECTION, None),
+                       (b.VAR_EUCLID, None), (b.VAR_REINFORCE, None), (b.VAR_GENERAL, [-1.0, 0.5, -2.0, lam, 0.0, 0.1])):
+        c = torch.empty(B, device="cuda")
+        info = torch.zeros(1, dtype=torch.int32, device="cuda")
+        lam_v = 1e-3 if variant == b.VAR_DIRECTION else lam
+        b.isopo_transform_advantages(Kd, Ad, variant, lam_v, c, info, g)
+        torch.cuda.synchronize()
+        pqr, regs = (tuple(g[:3]), tuple(np.float32(g[3:]).astype(np.float64))) if g else (None, None)
+        want = orc.transform_advantages(K.astype(np.float64), A.astype(np.float64), VARIANT_NAME[variant],
+                                        float(np.float32(lam_v)), pqr, regs)
+        assert rel_fro(c.cpu().numpy(), want) <= 1e-6, (B, variant)
+
+
+def test_not_pd_pivot_index_in_a_later_block(b):
+    B = 70
+    K = _gram(B, 2, 3).astype(np.float64)
+    K[40, 40] = -1.0  # leading minor of order 41 is not positive definite
+    Kd = torch.from_numpy(K.astype(np.float32)).cuda()
+    c = torch.empty(B, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.isopo_transform_advantages(Kd, torch.ones(B, device="cuda"), b.VAR_INTERACTING, 0.0, c, info)
+    torch.cuda.synchronize()
+    assert int(info.item()) == 41
