@@ -1,0 +1,256 @@
+// Gram route to the layer NTK on the tensor cores.
+//
+// Every token gradient is the rank-one matrix dY_t x_t^T (Eq. one / Eq. two), hence
+//   K_ij = sum_{t in i, s in j} (dY_t . dY_s)(x_t . x_s) = [ S ((dY dY^T) o (X X^T)) S^T ]_ij
+// with S the B x T sequence indicator.  For a pair of 128-token tiles (I <= J) this kernel forms
+// P = X_I X_J^T (contraction over d_in) and Q = dY_I dY_J^T (contraction over d_out) as two
+// 128 x 128 float32 accumulators in tensor memory, and its epilogue multiplies them elementwise and
+// adds the products into K by (sequence of row token, sequence of column token).  Neither T x T
+// matrix ever leaves the SM.
+//
+// Only token pairs t <= s are visited.  A pair t < s inside one sequence stands for (t,s) and
+// (s,t) and counts twice; a pair across sequences i < j lands in K_ij once (K_ji is mirrored at the
+// end); t = s counts once.
+//
+//   warp 0      TMA producer: [128 tokens] x [64 features] boxes of X then of dY, 6-stage ring
+//   warp 1      MMA issuer: tcgen05.mma 128 x 128 x 16, K-major operands
+//   warps 2-5   epilogue: tcgen05.ld of P and Q, product, segmented sums, float atomics into K
+#include "tc_common.cuh"
+
+namespace isopo {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kTT = 128;                       // tokens per tile
+constexpr int kKF = 64;                        // features per stage (128 bytes of bf16)
+constexpr int kStages = 6;
+constexpr int kOperandBytes = kTT * 128;       // 16 KB
+constexpr int kStageBytes = 2 * kOperandBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;            // 2 buffers x (P 128 + Q 128) columns
+
+struct GramParams {
+  const int32_t* tokseq;
+  float* K;
+  int64_t T;
+  int B, nT, d_in, d_out;
+  int32_t* info;
+};
+
+// u = J (J + 1) / 2 + I with I <= J
+__device__ __forceinline__ void decode_pair(long long u, int& I, int& J) {
+  long long j = (long long)((sqrt(8.0 * (double)u + 1.0) - 1.0) * 0.5);
+  while ((j + 1) * (j + 2) / 2 <= u) ++j;
+  while (j * (j + 1) / 2 > u) --j;
+  J = (int)j;
+  I = (int)(u - j * (j + 1) / 2);
+}
+
+__device__ __forceinline__ float warp_sum_f(float v) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Adds `v` (one value per lane, lane = tile row) into K[row_seq][col_seq]; one atomic per warp when
+// all rows of the warp belong to the same sequence.
+__device__ __forceinline__ void flush_segment(float* __restrict__ K, int B, int row_seq, int col_seq, float v) {
+  const unsigned same = __match_any_sync(0xffffffffu, row_seq);
+  if (same == 0xffffffffu) {
+    v = warp_sum_f(v);
+    if ((threadIdx.x & 31) == 0 && v != 0.f) atomicAdd(&K[(size_t)row_seq * B + col_seq], v);
+  } else if (v != 0.f) {
+    atomicAdd(&K[(size_t)row_seq * B + col_seq], v);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY, GramParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto accfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto accempty_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accfull_bar(b), 1); mbar_init(accempty_bar(b), 4); }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const long long total_units = (long long)p.nT * (p.nT + 1) / 2;
+  const int nkx = (p.d_in + kKF - 1) / kKF, nky = (p.d_out + kKF - 1) / kKF;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tensormap(&mapX);
+      prefetch_tensormap(&mapY);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        int I, J;
+        decode_pair(u, I, J);
+        const bool diag = I == J;
+        for (int kb = 0; kb < nkx + nky; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdGram))) break;
+          const CUtensorMap* map = kb < nkx ? &mapX : &mapY;
+          const int x = (kb < nkx ? kb : kb - nkx) * kKF;
+          const uint32_t dst = smem_base + stage * kStageBytes;
+          mbar_arrive_expect_tx(full_bar(stage), diag ? kOperandBytes : kStageBytes);
+          tma_load_2d(dst, map, x, I * kTT, full_bar(stage));
+          if (!diag) tma_load_2d(dst + kOperandBytes, map, x, J * kTT, full_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kTT, kTT, false, false);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        int I, J;
+        decode_pair(u, I, J);
+        const bool diag = I == J;
+        if (!(ok = mbar_wait(accempty_bar(acc), acc_phase ^ 1u, abort_flag, p.info, kIdGram))) break;
+        tc_fence_after_sync();
+        for (int kb = 0; kb < nkx + nky; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.info, kIdGram))) break;
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_base + stage * kStageBytes;
+          const uint32_t b_addr = diag ? a_addr : a_addr + kOperandBytes;
+          const bool second = kb >= nkx;  // accumulating Q
+          const uint32_t d_tmem = tmem_base + (uint32_t)acc * 256 + (second ? 128u : 0u);
+          const int kk = second ? kb - nkx : kb;
+#pragma unroll
+          for (int k16 = 0; k16 < kKF / 16; ++k16) {
+            const uint64_t a_desc = make_sdesc_sw128(a_addr + k16 * 32, 16, 1024);
+            const uint64_t b_desc = make_sdesc_sw128(b_addr + k16 * 32, 16, 1024);
+            mma_bf16(d_tmem, a_desc, b_desc, idesc, (kk | k16) != 0);
+          }
+          mma_commit(empty_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        mma_commit(accfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    const int q = warp & 3, row = q * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (long long u = blockIdx.x; u < total_units; u += gridDim.x) {
+      int I, J;
+      decode_pair(u, I, J);
+      const bool diag = I == J;
+      // sequence of this thread's row token and of every column token (clamped past the end; those
+      // rows and columns are zero in P and Q)
+      const int64_t trow = (int64_t)I * kTT + row;
+      const int row_seq = __ldg(p.tokseq + min(trow, p.T - 1));
+      int csr[4];  // csr[g] of lane l = sequence of column token 32 g + l
+#pragma unroll
+      for (int g = 0; g < 4; ++g) csr[g] = __ldg(p.tokseq + min((int64_t)J * kTT + g * 32 + lane, p.T - 1));
+      if (!mbar_wait(accfull_bar(acc), acc_phase, abort_flag, p.info, kIdGram)) break;
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * 256;
+      int cur = __shfl_sync(0xffffffffu, csr[0], 0);
+      float wseg = row_seq == cur ? 2.f : 1.f, run = 0.f;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const int c0 = g * 32;
+        uint32_t pv[32], qv[32];
+        tmem_ld32(taddr + c0, pv);
+        tmem_ld32(taddr + 128 + c0, qv);
+        tmem_ld_wait();
+        const bool one_segment = __shfl_sync(0xffffffffu, csr[g], 31) == cur;  // column sequences never decrease
+        if (one_segment && !diag) {
+          float s = 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) s = fmaf(__uint_as_float(pv[e]), __uint_as_float(qv[e]), s);
+          run = fmaf(wseg, s, run);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int c = c0 + e, sc = __shfl_sync(0xffffffffu, csr[g], e);
+            if (sc != cur) {  // uniform across the warp
+              flush_segment(p.K, p.B, row_seq, cur, run);
+              run = 0.f;
+              cur = sc;
+              wseg = row_seq == cur ? 2.f : 1.f;
+            }
+            const float h = __uint_as_float(pv[e]) * __uint_as_float(qv[e]);
+            const float f = (!diag || c > row) ? wseg : (c == row ? 1.f : 0.f);
+            run = fmaf(f, h, run);
+          }
+        }
+      }
+      flush_segment(p.K, p.B, row_seq, cur, run);
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(accempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  if (*abort_flag) __nanosleep(100000);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+__global__ void k_mirror_upper_gram(float* __restrict__ K, int B) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= B * B) return;
+  const int i = e / B, j = e % B;
+  if (j < i) K[e] = K[(size_t)j * B + i];
+}
+
+}  // namespace
+
+isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
+                       float* K, int32_t* info, cudaStream_t st) {
+  CUtensorMap mapX, mapY;
+  isopo_status s = make_map_2d_bf16(&mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kTT);
+  if (s != ISOPO_OK) return s;
+  s = make_map_2d_bf16(&mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kTT);
+  if (s != ISOPO_OK) return s;
+  int dev = 0, sms = 0;
+  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
+  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_gram, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
+  GramParams p{tokseq, K, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info};
+  const long long units = (long long)p.nT * (p.nT + 1) / 2;
+  const int grid = (int)std::min<long long>(units, sms);
+  {
+    LaunchScope scope(kIdGram, st);
+    k_bf16_gram<<<grid, kThreads, kSmemBytes, st>>>(mapX, mapY, p);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  {
+    LaunchScope scope(kIdMirror, st);
+    k_mirror_upper_gram<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+}  // namespace isopo

@@ -12,6 +12,12 @@
 //               zeroes the token rows past the end of the sequence in the last slab
 //   warps 2-5   epilogue: TMEM -> registers -> bf16 (round to nearest even) -> workspace
 //
+// The same pipeline, instantiated with kFolded = true, is the stand-alone weight-gradient GEMM
+// dW = (c_seq(t) dY)^T X (Alg. 1 "grad += advantages * rescaled gradient"): its work units are
+// (tile, token slab), four extra warps multiply every dY row of a landed stage by its sequence's
+// coefficient in shared memory (round to nearest even) before the MMA warp may read it, and the
+// epilogue adds float32 tiles into the row-major dW.
+//
 // Stored layout of one tile (64 KB, private to the library): element (m, n) of the tile sits at
 // ((n / 8) * 128 + m) * 8 + n % 8, so that a warp's 32 rows write 512 contiguous bytes.
 #include "tc_common.cuh"
@@ -30,6 +36,7 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kChunkBytes = kKB * 128;                 // one [64 tokens][64 cols] box
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 192;
+constexpr int kThreadsFolded = 320;                    // + 4 warps that scale the dY rows
 constexpr uint32_t kTmemCols = 512;                    // two 256-column float32 accumulators
 
 struct SeqGradParams {
@@ -38,9 +45,32 @@ struct SeqGradParams {
   int64_t n_pad;
   int B, tiles_m, tiles_n;
   int32_t* info;
+  // folded weight-gradient GEMM only
+  const float* coeffs;
+  const int32_t* tokseq;
+  float* dW;
+  int64_t T, slab;  // tokens per work unit (a multiple of 64)
+  int nslabs, d_in, d_out;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+// Work unit u -> (token range, tile).  Per-sequence mode: sequence-major, u = i * tiles + tile.
+// Folded mode: u = slab * tiles + tile.
+template <bool kFolded>
+__device__ __forceinline__ void decode_unit(const SeqGradParams& p, long long u, int tiles, int& tile, int64_t& t0,
+                                            int64_t& t1, int& seq) {
+  seq = (int)(u / tiles);
+  tile = (int)(u % tiles);
+  if (kFolded) {
+    t0 = (int64_t)seq * p.slab;
+    t1 = min(p.T, t0 + p.slab);
+  } else {
+    t0 = p.off[seq];
+    t1 = p.off[seq + 1];
+  }
+}
+
+template <bool kFolded>
+__global__ void __launch_bounds__(kFolded ? kThreadsFolded : kThreads, 1)
 k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapX, SeqGradParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -51,12 +81,17 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto accfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
   auto accempty_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  auto scaled_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 4 + s); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kStages + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+      mbar_init(scaled_bar(s), 4);
+    }
     for (int b = 0; b < 2; ++b) { mbar_init(accfull_bar(b), 1); mbar_init(accempty_bar(b), 4); }
     *abort_flag = 0;
     fence_barrier_init();
@@ -68,7 +103,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
 
   const int tiles_per_seq = p.tiles_m * p.tiles_n;
-  const long long total_units = (long long)p.B * tiles_per_seq;
+  const long long total_units = (long long)(kFolded ? p.nslabs : p.B) * tiles_per_seq;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -79,9 +114,10 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
       uint32_t phase = 0;
       bool ok = true;
       for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-        const int i = (int)(u / tiles_per_seq), tile = (int)(u % tiles_per_seq);
+        int i, tile;
+        int64_t t0, t1;
+        decode_unit<kFolded>(p, u, tiles_per_seq, tile, t0, t1, i);
         const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
-        const int64_t t0 = p.off[i], t1 = p.off[i + 1];
         const int nkb = (int)((t1 - t0 + kKB - 1) / kKB);
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdSeqGrad))) break;
@@ -105,20 +141,23 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
     uint32_t phase = 0, acc_phase = 0;
     bool ok = true;
     for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-      const int i = (int)(u / tiles_per_seq);
-      const int64_t t0 = p.off[i], t1 = p.off[i + 1];
+      int i, tile;
+      int64_t t0, t1;
+      decode_unit<kFolded>(p, u, tiles_per_seq, tile, t0, t1, i);
       const int len = (int)(t1 - t0);
       const int nkb = (len + kKB - 1) / kKB;
       if (!(ok = mbar_wait(accempty_bar(acc), acc_phase ^ 1u, abort_flag, p.info, kIdSeqGrad))) break;
       tc_fence_after_sync();
       const uint32_t d_tmem = tmem_base + (uint32_t)acc * kTileN;
       for (int kb = 0; kb < nkb; ++kb) {
-        if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.info, kIdSeqGrad))) break;
+        // folded mode: the scaler warps hand the stage over (they have waited for the TMA bytes)
+        if (!(ok = mbar_wait(kFolded ? scaled_bar(stage) : full_bar(stage), phase, abort_flag, p.info, kIdSeqGrad)))
+          break;
         tc_fence_after_sync();
         const uint32_t a_addr = smem_base + stage * kStageBytes, b_addr = a_addr + kABytes;
-        const int valid = min(kKB, len - kb * kKB);  // token rows of this slab that belong to sequence i
+        const int valid = min(kKB, len - kb * kKB);  // token rows of this slab that belong to the unit
         const int n16 = (valid + 15) >> 4;           // 16-token MMA steps that hold any of them
-        if (valid < n16 * 16) {
+        if (!kFolded && valid < n16 * 16) {
           // rows [valid, n16*16) hold the next sequence's tokens: zero them in the dY tile
           const int nbytes = (n16 * 16 - valid) * 128;
 #pragma unroll
@@ -146,7 +185,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
       __syncwarp();
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-  } else {
+  } else if (warp < 6) {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const int row = q * 32 + lane;
@@ -156,27 +195,89 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
       const int i = (int)(u / tiles_per_seq), tile = (int)(u % tiles_per_seq);
       if (!mbar_wait(accfull_bar(acc), acc_phase, abort_flag, p.info, kIdSeqGrad)) break;
       tc_fence_after_sync();
-      uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)i * p.n_pad + (size_t)tile * kTileElems) + row;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTileN;
+      if (!kFolded) {
+        uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)i * p.n_pad + (size_t)tile * kTileElems) + row;
 #pragma unroll 2
-      for (int jc = 0; jc < kTileN / 32; ++jc) {
-        uint32_t r[32];
-        tmem_ld32(taddr + jc * 32, r);
-        tmem_ld_wait();
+        for (int jc = 0; jc < kTileN / 32; ++jc) {
+          uint32_t r[32];
+          tmem_ld32(taddr + jc * 32, r);
+          tmem_ld_wait();
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          uint4 o;
-          o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-          o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-          o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-          o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-          dst[(size_t)(jc * 4 + v) * kTileM] = o;
+          for (int v = 0; v < 4; ++v) {
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+            o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+            o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+            o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+            dst[(size_t)(jc * 4 + v) * kTileM] = o;
+          }
+        }
+      } else {
+        // dW[m, n0 .. n0+255] += accumulator row; token slabs of one tile meet here, hence atomics
+        const int m = (tile / p.tiles_n) * kTileM + row, n0 = (tile % p.tiles_n) * kTileN;
+        float* dst = p.dW + (size_t)m * p.d_in + n0;
+#pragma unroll 2
+        for (int jc = 0; jc < kTileN / 32; ++jc) {
+          uint32_t r[32];
+          tmem_ld32(taddr + jc * 32, r);
+          tmem_ld_wait();
+          if (m < p.d_out) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              const int n = n0 + jc * 32 + v * 4;
+              if (n < p.d_in)  // d_in is a multiple of 8, so a group of 4 is all in or all out
+                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + jc * 32 + v * 4),
+                             "f"(__uint_as_float(r[v * 4 + 0])), "f"(__uint_as_float(r[v * 4 + 1])),
+                             "f"(__uint_as_float(r[v * 4 + 2])), "f"(__uint_as_float(r[v * 4 + 3]))
+                             : "memory");
+            }
+          }
         }
       }
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(accempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else if (kFolded) {
+    // ------------------------------------------------------------------ scaler (warps 6..9)
+    // Thread (r, h): token row r of the stage, half h of each 128-byte row, in both dY chunks.
+    // The 128-byte swizzle permutes 16-byte pieces inside a row only, so a whole row can be scaled
+    // in place without knowing the permutation.
+    const int st = threadIdx.x - 192, r = st >> 1, h = st & 1;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      int i, tile;
+      int64_t t0, t1;
+      decode_unit<kFolded>(p, u, tiles_per_seq, tile, t0, t1, i);
+      const int nkb = (int)((t1 - t0 + kKB - 1) / kKB);
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int64_t t = t0 + (int64_t)kb * kKB + r;
+        const float c = t < t1 ? __ldg(p.coeffs + __ldg(p.tokseq + t)) : 0.f;
+        if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.info, kIdSeqGrad))) break;
+        const uint32_t a_addr = smem_base + stage * kStageBytes + r * 128 + h * 64;
+#pragma unroll
+        for (int ch = 0; ch < kTileM / 64; ++ch)
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            const uint32_t addr = a_addr + ch * kChunkBytes + v * 16;
+            uint32_t w[4];
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr) : "memory");
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              w[e] = pack_bf16x2(c * __uint_as_float(w[e] << 16), c * __uint_as_float(w[e] & 0xffff0000u));
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                         "r"(w[3]) : "memory");
+          }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(scaled_bar(stage));
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
     }
   }
 
@@ -189,24 +290,67 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
 
 }  // namespace
 
+static isopo_status make_maps(CUtensorMap* mapY, CUtensorMap* mapX, const void* X, const void* dY, int64_t T, int d_in,
+                              int d_out) {
+  isopo_status s = make_map_2d_bf16(mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kKB);
+  if (s != ISOPO_OK) return s;
+  return make_map_2d_bf16(mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kKB);
+}
+
+static isopo_status sm_count(int* sms) {
+  int dev = 0;
+  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
+  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev));
+  return ISOPO_OK;
+}
+
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
                            const int64_t* off_dev, int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st) {
   (void)off_host;
   CUtensorMap mapY, mapX;
-  isopo_status s = make_map_2d_bf16(&mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kKB);
+  isopo_status s = make_maps(&mapY, &mapX, X, dY, T, d_in, d_out);
   if (s != ISOPO_OK) return s;
-  s = make_map_2d_bf16(&mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kKB);
-  if (s != ISOPO_OK) return s;
-  int dev = 0, sms = 0;
-  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
-  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  SeqGradParams p{off_dev, (__nv_bfloat16*)G, L.n_pad, B, L.tiles_m, L.tiles_n, info};
+  int sms = 0;
+  if ((s = sm_count(&sms)) != ISOPO_OK) return s;
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  SeqGradParams p{};
+  p.off = off_dev; p.G = (__nv_bfloat16*)G; p.n_pad = L.n_pad; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
+  p.info = info;
   const long long units = (long long)B * L.tiles_m * L.tiles_n;
   const int grid = (int)std::min<long long>(units, sms);
   {
     LaunchScope scope(kIdSeqGrad, st);
-    k_bf16_seq_grad<<<grid, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
+    k_bf16_seq_grad<false><<<grid, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* coeffs,
+                              const int32_t* tokseq, float* dW, float beta, int32_t* info, cudaStream_t st) {
+  CUtensorMap mapY, mapX;
+  isopo_status s = make_maps(&mapY, &mapX, X, dY, T, d_in, d_out);
+  if (s != ISOPO_OK) return s;
+  int sms = 0;
+  if ((s = sm_count(&sms)) != ISOPO_OK) return s;
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  if (beta == 0.f) ISOPO_CUDA_TRY(cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)d_in * d_out, st));
+  SeqGradParams p{};
+  p.tiles_m = (d_out + kTileM - 1) / kTileM;
+  p.tiles_n = (d_in + kTileN - 1) / kTileN;
+  p.info = info; p.coeffs = coeffs; p.tokseq = tokseq; p.dW = dW; p.T = T; p.d_in = d_in; p.d_out = d_out;
+  // token slabs: enough (tile, slab) units to fill the machine about twice, each slab a multiple of 64 tokens
+  const long long tiles = (long long)p.tiles_m * p.tiles_n;
+  const long long kblocks = (T + kKB - 1) / kKB;
+  long long nslabs = std::max<long long>(1, std::min<long long>(kblocks, (2ll * sms + tiles - 1) / tiles));
+  const long long kb_per = (kblocks + nslabs - 1) / nslabs;
+  nslabs = (kblocks + kb_per - 1) / kb_per;
+  p.slab = kb_per * kKB;
+  p.nslabs = (int)nslabs;
+  const int grid = (int)std::min<long long>(tiles * nslabs, sms);
+  {
+    LaunchScope scope(kIdWeightGrad, st);
+    k_bf16_seq_grad<true><<<grid, kThreadsFolded, kSmemBytes, st>>>(mapY, mapX, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
