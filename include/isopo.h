@@ -159,6 +159,38 @@ ISOPO_API isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dt
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_layer_gram_static: isopo_layer_gram on the GRAM route without a caller workspace and
+ * without any allocation (the paper has no counterpart; this exists for the way the library gets
+ * embedded).
+ *
+ * Who needs it: callers that may not allocate device memory where the layer hook runs - a hook
+ * inside a framework whose caching allocator owns the device and rejects raw cudaMalloc, code that
+ * runs while that allocator is locked, or an embedder that gave the whole device to another pool.
+ * The scratch the route needs (device copy of the offsets, token -> sequence map, float64
+ * accumulators of the float32 route) lives in a fixed array inside the library's device image:
+ * about 0.8 MB that every GPU which loads the library keeps reserved until the process exits.
+ *
+ * Limits: T <= ISOPO_STATIC_MAX_TOKENS and B <= ISOPO_STATIC_MAX_SEQS; larger problems return
+ * ISOPO_ERR_UNSUPPORTED (isopo_last_cuda_error() then says why) and must use isopo_layer_gram.
+ * The call makes no cudaMalloc / cudaFree and calls no allocating routine; event timing
+ * (isopo_profile_enable) is suspended for its duration.
+ *
+ * The first call on each device looks up the array's device address (one cudaGetSymbolAddress with
+ * that device current); make that first call outside any stream capture.  All calls on a device
+ * share the one array: calls whose kernels could overlap on the GPU (different streams, no
+ * ordering between them) race on it and must be serialised by the caller.  The array keeps what
+ * the previous call left; every part that is read is rewritten or cleared first.
+ *
+ * Arguments and the result are those of isopo_layer_gram with path = ISOPO_PATH_GRAM; K agrees
+ * with it up to the order of the float atomic additions.
+ */
+#define ISOPO_STATIC_MAX_TOKENS 65536
+#define ISOPO_STATIC_MAX_SEQS 256
+ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in,
+                                               int d_out, const int64_t* seq_offsets_host, int B, float* K,
+                                               int32_t* info, void* cuda_stream);
+
+/*
  * Measurement hooks (the paper has no counterpart).  While enabled, every kernel the library
  * launches is bracketed by CUDA events on its stream.  isopo_profile_collect synchronises those
  * events, adds the elapsed milliseconds and launch counts per kernel into the caller's arrays

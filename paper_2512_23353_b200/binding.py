@@ -26,8 +26,9 @@ INFO_TIMEOUT = 0x40000000
 EXPORTS = (
     "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",
     "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad",
-    "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name",
+    "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
 )
+STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
 NUM_KERNELS = 13
 
 
@@ -62,6 +63,9 @@ def _load():
     lib.isopo_weight_grad.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
                                       c.c_void_p, c.c_int, c.c_int, c.c_void_p, c.c_float, c.c_void_p, c.c_size_t,
                                       c.c_void_p, c.c_void_p]
+    lib.isopo_layer_gram_static.restype = c.c_int
+    lib.isopo_layer_gram_static.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
+                                            c.c_int, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.isopo_profile_enable.restype = None
     lib.isopo_profile_enable.argtypes = [c.c_int]
     lib.isopo_profile_collect.restype = c.c_int
@@ -130,6 +134,22 @@ def isopo_layer_gram(X: torch.Tensor, dY: torch.Tensor, seq_offsets, K: torch.Te
                               off.ctypes.data, B, path, K.data_ptr(), ws.data_ptr(), ws.numel(), info.data_ptr(),
                               _stream())
     _check(st, "isopo_layer_gram")
+
+
+def isopo_layer_gram_static(X: torch.Tensor, dY: torch.Tensor, seq_offsets, K: torch.Tensor,
+                            info: torch.Tensor) -> None:
+    """isopo_layer_gram on the Gram route for callers that cannot allocate: the scratch is a fixed
+    array inside the library (at most STATIC_MAX_TOKENS tokens and STATIC_MAX_SEQS sequences).
+    Calls on one device share that array, so do not let two of them overlap on the GPU."""
+    off = _offsets(seq_offsets)
+    B = off.shape[0] - 1
+    assert X.is_cuda and dY.is_cuda and X.is_contiguous() and dY.is_contiguous() and X.dtype == dY.dtype
+    assert K.dtype == torch.float32 and K.is_contiguous() and K.numel() == B * B and info.dtype == torch.int32
+    st = lib.isopo_layer_gram_static(X.data_ptr(), dY.data_ptr(), _dtype_code(X), X.shape[0], X.shape[1],
+                                     dY.shape[1], off.ctypes.data, B, K.data_ptr(), info.data_ptr(), _stream())
+    if st == ERR_UNSUPPORTED:
+        raise IsopoError(st, f"isopo_layer_gram_static: ISOPO_ERR_UNSUPPORTED [{lib.isopo_last_cuda_error().decode()}]")
+    _check(st, "isopo_layer_gram_static")
 
 
 def isopo_transform_advantages(K: torch.Tensor, A: torch.Tensor, variant: int, lam: float, coeffs: torch.Tensor,

@@ -12,7 +12,10 @@ namespace isopo {
 static thread_local char g_cuda_err[256] = "no error";
 
 void set_cuda_error(cudaError_t e, const char* where) {
-  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
+  if (e == cudaSuccess)
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s", where);  // a plain explanation, no CUDA error behind it
+  else
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
 }
 
 // ---- measurement hooks ----
@@ -46,6 +49,9 @@ LaunchScope::LaunchScope(int id, cudaStream_t st) : slot_(-1), st_(st) {
 LaunchScope::~LaunchScope() {
   if (slot_ >= 0) cudaEventRecord(g_prof[slot_].b, st_);
 }
+
+ProfilingPause::ProfilingPause() : was_on_(g_prof_on) { g_prof_on = false; }
+ProfilingPause::~ProfilingPause() { g_prof_on = was_on_; }
 
 WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path resolved) {
   WsLayout L{};

@@ -45,6 +45,16 @@ class LaunchScope {
   cudaStream_t st_;
 };
 
+// Suspends event timing for the lifetime of the object (launch counting continues).
+class ProfilingPause {
+ public:
+  ProfilingPause();
+  ~ProfilingPause();
+
+ private:
+  bool was_on_;
+};
+
 struct WsLayout {
   size_t off_offsets;  // int64 [B+1]
   size_t off_tokseq;   // int32 [T]
