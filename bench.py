@@ -109,6 +109,29 @@ def dist_env():
     return rank, world, local
 
 
+def rank_workload(w, rank: int, world: int):
+    """The microbatch recipe of one rank: the path shards by independent microbatches (K is defined
+    per microbatch), so with several ranks each draws its own from a rank-dependent seed."""
+    if world == 1:
+        return w
+    from dataclasses import replace
+    return replace(w, seed=w.seed + 7919 * rank)
+
+
+def reduce_over_ranks(elapsed_ms: float, tokens: float, device=None):
+    """(max elapsed over ranks, total tokens over ranks); identity without a process group."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return elapsed_ms, tokens
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([tokens], dtype=torch.float64, device=device)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(n.item())
+
+
 # ------------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ------------------------------------------------------------------------------------------------
@@ -194,18 +217,20 @@ def run_gpu(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    w = wl.WORKLOADS[args.workload]
-    if world > 1:  # every rank its own microbatch
-        from dataclasses import replace
-        w = replace(w, seed=w.seed + 7919 * rank)
+    w = rank_workload(wl.WORKLOADS[args.workload], rank, world)
     off, A_host = wl.microbatch(w)
-    T, B = int(off[-1]), w.B
+    if args.seqs:  # profiling aid: the first --seqs sequences only (keeps an ncu capture small)
+        off, A_host = off[: args.seqs + 1].copy(), A_host[: args.seqs].copy()
+    T, B = int(off[-1]), len(A_host)
+    wanted = set(args.layers.split(",")) if args.layers else None
+    w_layers = [l for l in w.layers if wanted is None or l.name in wanted]
+    n_warm = args.warmup if args.short_warmup else max(args.warmup, 3)
     dt_code = b.BF16 if w.dtype == "bf16" else b.F32
     variant = b.VAR_INTERACTING if args.variant == "interacting" else b.VAR_NORMALISED
 
     layers = []
     ws_bytes = 0
-    for layer in w.layers:
+    for layer in w_layers:
         X, dY = wl.layer_inputs_device(w, layer, T, dev)
         path = b.isopo_choose_path(dt_code, T, layer.d_in, layer.d_out, B)
         ws_bytes = max(ws_bytes, b.isopo_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, path))
@@ -232,7 +257,7 @@ def run_gpu(args):
     torch.cuda.synchronize()
     for L in layers:
         L["lam"] = 1e-3 * float(torch.diagonal(L["K"]).mean().item())
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(n_warm):
         step()
     torch.cuda.synchronize()
     if int(info.item()) != 0:
@@ -261,15 +286,7 @@ def run_gpu(args):
     prof = b.isopo_profile_collect()
     if int(info.item()) != 0:
         raise SystemExit(f"device-side error during the timed region: info={int(info.item()):#x}")
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-        tok = torch.tensor([T], dtype=torch.float64, device=dev)
-        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
-        total_tokens = float(tok.item())
-    else:
-        total_tokens = float(T)
+    elapsed_ms, total_tokens = reduce_over_ranks(elapsed_ms, float(T), dev)
     ms_per_step = elapsed_ms / args.steps
     value = total_tokens / (ms_per_step / 1000.0)
 
@@ -368,7 +385,7 @@ def run_gpu(args):
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "B": B, "tokens": T, "variant": args.variant,
                    "layers": [f"{L['layer'].name}:{L['layer'].d_in}->{L['layer'].d_out}" for L in layers],
@@ -401,6 +418,9 @@ def main():
     ap.add_argument("--variant", default="interacting", choices=["interacting", "normalised"])
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--layers", default="", help="comma-separated projection names (default: all of the block)")
+    ap.add_argument("--seqs", type=int, default=0, help="use only the first N sequences (profiling aid)")
+    ap.add_argument("--short-warmup", action="store_true", help="allow fewer than 3 warm-up steps (profiling only)")
     ap.add_argument("--cpu-seqs", type=int, default=8)
     ap.add_argument("--cpu-len-div", type=int, default=8)
     args = ap.parse_args()
