@@ -19,7 +19,6 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -48,58 +47,66 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU through NVML (every 5 ms, in a thread)
+    while the timed region runs."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
-        self.proc = None
-        self.lines = []
+    def __init__(self, cuda_index: int):
+        self.cuda_index = cuda_index
+        self.samples = []
+        self.stop_flag = threading.Event()
+        self.thread = None
+        self.error = None
+
+    def _handle(self, nv):
+        import torch
+        props = torch.cuda.get_device_properties(self.cuda_index)
+        try:
+            bus = f"{props.pci_domain_id:08x}:{props.pci_bus_id:02x}:{props.pci_device_id:02x}.0"
+            return nv.nvmlDeviceGetHandleByPciBusId(bus.encode())
+        except Exception:
+            return nv.nvmlDeviceGetHandleByIndex(self.cuda_index)
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._pump, daemon=True)
-            self.thread.start()
-        except OSError:
-            self.proc = None
+            import pynvml as nv
+            nv.nvmlInit()
+            h = self._handle(nv)
+            reasons_fn = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+            smax = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+        except Exception as e:  # no NVML: the bench line says so instead of inventing clocks
+            self.error = f"NVML unavailable: {e}"
+            return
 
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+        def pump():
+            while not self.stop_flag.is_set():
+                try:
+                    self.samples.append((nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM), smax,
+                                         nv.nvmlDeviceGetPowerUsage(h) / 1000.0, int(reasons_fn(h))))
+                except Exception:
+                    pass
+                time.sleep(0.005)
+
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, smax, power, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [x.strip() for x in ln.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                smax.append(float(parts[1]))
-                power.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        if not sm:
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [self.error or "no samples"]}
+        self.stop_flag.set()
+        self.thread.join(timeout=2)
+        if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "power_w_max": max(power),
-                "samples": len(sm), "reasons": sorted(reasons)}
+        sm = [x[0] for x in self.samples]
+        mask = 0
+        for x in self.samples:
+            mask |= x[3]
+        return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": self.samples[0][1],
+                "power_w_max": max(x[2] for x in self.samples), "samples": len(sm),
+                "reasons": sorted(name for bit, name in self.REASONS.items() if mask & bit)}
 
 
 def dist_env():
@@ -324,8 +331,20 @@ def run_gpu(args):
             kernels[name]["hbm_gbs"] = g_bytes / (kernels[name]["ms_per_step"] * 1e-3) / 1e9
             kernels[name]["hbm_frac"] = kernels[name]["hbm_gbs"] / peaks["hbm_gbs"]
 
+    # ---- per-projection breakdown (one more untimed pass, events per kernel) ----
+    per_layer = []
+    b.isopo_profile_enable(True)
+    for L in layers:
+        b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
+        b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
+        b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+        pl = b.isopo_profile_collect()
+        per_layer.append({"layer": L["layer"].name, **{k: round(v[0], 4) for k, v in pl.items()}})
+    b.isopo_profile_enable(False)
+
     # ---- plain dW GEMM (cuBLAS through torch) on the same inputs, same run ----
     plain_ms = 0.0
+    plain_by_layer = []
     for L in layers:
         for _ in range(3):
             torch.matmul(L["dY"].t(), L["X"])
@@ -336,7 +355,8 @@ def run_gpu(args):
             torch.matmul(L["dY"].t(), L["X"])
         c.record()
         torch.cuda.synchronize()
-        plain_ms += a.elapsed_time(c) / args.steps
+        plain_by_layer.append(a.elapsed_time(c) / args.steps)
+        plain_ms += plain_by_layer[-1]
     overhead = ms_per_step / plain_ms
 
     # ---- end to end: host buffers, copies inside the timed region ----
@@ -402,6 +422,7 @@ def run_gpu(args):
         "plain_dw_gemm_ms": plain_ms,
         "overhead_vs_plain_dw_gemm": overhead,
         "kernels": kernels,
+        "per_layer_ms": [dict(pl, plain_dw_gemm=round(pm, 4)) for pl, pm in zip(per_layer, plain_by_layer)],
     }
     print(json.dumps(out))
     if world > 1:
@@ -411,7 +432,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llm_1p5b")

@@ -96,6 +96,8 @@ isopo_status f32_weight_grad(const float* X, const float* dY, int64_t T, int d_i
 // bf16 tcgen05 path
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
                            const int64_t* off_dev, int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st);
+isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
+                                int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st);
 isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t* info, cudaStream_t st);
 isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
                           float beta, cudaStream_t st);

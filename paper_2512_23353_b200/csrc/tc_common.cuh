@@ -14,6 +14,27 @@ namespace isopo {
 namespace tc {
 
 // ---------------------------------------------------------------------------------------------
+// Stored per-sequence gradients (bf16, materialised route; the order is private to the library).
+//
+// G_i is cut into 128 x 256 tiles (tile = tile_m * tiles_n + tile_n) and every tile into "pieces" of
+// 32 rows x 8 columns = 256 elements = 512 bytes: piece (tile, j, q) holds rows 32q .. 32q+31 and
+// columns 8j .. 8j+7 of the tile, row-major inside (row r at 16-byte slot r % 32).  That is exactly
+// what one epilogue warp writes with one 16-byte store per lane.  Pieces are the OUTER index and
+// the sequence the inner one:
+//     uint4 index of (piece p, sequence i, slot l) = (p * B + i) * 32 + l,   p = (tile * 32 + j) * 4 + q
+// so the B copies of one piece are contiguous (B x 512 bytes).  The NTK kernel contracts over
+// pieces and reads each such block once, front to back; the combine kernel sums over i inside it.
+// Any fixed order of the elements of G_i gives the same <G_i, G_j>.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPieceElems = 256;
+__host__ __device__ __forceinline__ size_t stored_piece(int tile, int j, int q) {
+  return ((size_t)tile * 32 + (size_t)j) * 4 + (size_t)q;
+}
+__host__ __device__ __forceinline__ size_t stored_slot(size_t piece, int i, int B, int l) {
+  return (piece * (size_t)B + (size_t)i) * 32 + (size_t)l;
+}
+
+// ---------------------------------------------------------------------------------------------
 // host: tensor maps
 // ---------------------------------------------------------------------------------------------
 
@@ -22,6 +43,11 @@ namespace tc {
 // box_cols * 2 bytes must be 128.  Out-of-range elements read as zero.
 isopo_status make_map_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_elems,
                               uint32_t box_cols, uint32_t box_rows);
+
+// Stored per-sequence gradients viewed as (x = element inside a 256-element piece row, y = sequence,
+// z = piece): boxes of 64 elements x `box_rows` sequences x 1 piece, 128-byte swizzle.  Sequences
+// past B read as zero.
+isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows);
 
 // ---------------------------------------------------------------------------------------------
 // device: generic helpers
@@ -57,6 +83,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// One look at the barrier, never blocks.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Gives up after ~2^31 clock ticks (about a second) or as soon as another role of
 // this CTA has given up (`*abort_flag` != 0, shared memory); records ISOPO_INFO_TIMEOUT | code in
 // *info (only over a zero) and returns false.  Callers leave their loops and fall through to the
@@ -85,6 +122,20 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
 __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+// As tma_load_2d inside a CTA pair: the barrier may live in the other CTA of the pair (`bar` is a
+// shared::cluster address); the data still lands in this CTA.  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
@@ -131,6 +182,91 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- CTA pairs (cluster of two CTAs driving one 2-CTA tcgen05.mma) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {  // every thread of both CTAs
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrival that publishes this thread's earlier shared-memory writes to the whole pair (slow: keep it
+// out of per-stage loops)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// arrival that publishes nothing but "done" (e.g. a drained accumulator): CTA-scope release, cheap
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait inside a CTA pair.  kClusterAcquire: acquire at cluster scope, for the one case where
+// the arrival publishes the peer's ordinary shared-memory writes; completions of TMA copies and of
+// tcgen05.commit, and arrivals that only hand over tensor memory, need the CTA-scope form, which is
+// much cheaper in the MMA issuer's loop.  On giving up it also raises the peer's abort flag (`peer_abort`, a shared::cluster address) so that both
+// CTAs of the pair head for the teardown.
+template <bool kClusterAcquire = false>
+__device__ __forceinline__ bool mbar_wait_pair(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               uint32_t peer_abort, int32_t* info, int code) {
+  auto try_wait = [&]() { return kClusterAcquire ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+  if (try_wait()) return true;
+  const long long start = clock64();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (try_wait()) return true;
+    if (*abort_flag) return false;
+    if (clock64() - start > (1ll << 31)) {
+      *abort_flag = 1;
+      st_cluster_u32(peer_abort, 1u);
+      atomicCAS(info, 0, ISOPO_INFO_TIMEOUT | code);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t ncols) {  // one full warp in EACH CTA
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {  // one full warp in EACH CTA
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// 2-CTA MMA, issued by ONE thread of the pair's first CTA: each CTA supplies its half of A's rows
+// and of B's rows (same shared-memory offsets in both) and receives its half of D's rows.
+__device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              bool accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair once every MMA
+// issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3)
+      : "memory");
+}
 
 // ---- descriptors ----
 // Instruction descriptor, kind::f16 with bf16 A and B, float32 D.  a_mn / b_mn: operand is stored

@@ -97,7 +97,7 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
   const int nkx = (p.d_in + kKF - 1) / kKF, nky = (p.d_out + kKF - 1) / kKF;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       prefetch_tensormap(&mapX);
       prefetch_tensormap(&mapY);
       int stage = 0;
@@ -120,7 +120,7 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {  // elected, not "lane 0": lets the compiler keep the MMA operands in uniform registers
       constexpr uint32_t idesc = make_idesc_bf16(kTT, kTT, false, false);
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;

@@ -1,14 +1,15 @@
 // K = G_flat G_flat^T from the stored per-sequence gradients (Alg. 2 "make neural tangent kernel":
 // K_ij = sum(G_i * G_j)), and dW = sum_i c_i G_i from the same store (Alg. 2 last line).
 //
-// k_bf16_ntk: the B <= 256 stored gradients are the rows of a [B, n_pad] bf16 matrix.  Each CTA takes a
-// contiguous slab of the long contraction dimension, streams [B rows] x [64 elements] boxes through
-// a TMA ring, and uses every box as BOTH tcgen05 operands (K-major): rows 0..127 against all rows,
+// k_bf16_ntk: the B <= 256 stored gradients form a [pieces][B][256] bf16 array (tc_common.cuh).  Each CTA
+// takes a contiguous run of the long contraction dimension, streams [B rows] x [64 elements] boxes
+// (four per piece, so a CTA walks memory front to back) through a TMA ring, and uses every box as BOTH tcgen05 operands (K-major): rows 0..127 against all rows,
 // then rows 128..255 against rows 128..255 (the lower-left block is the mirror of the upper-right).
 // The float32 accumulators stay in tensor memory for the whole slab and are added into K once, with
 // reductions across CTAs by float atomics; a last tiny kernel mirrors the upper triangle.
 //
-// k_bf16_combine: pure streaming, one 16-byte chunk of every G_i per thread.
+// k_bf16_combine: pure streaming, one 16-byte slot of every G_i per thread; a warp reads 512
+// contiguous bytes per sequence and the B sequences of a piece back to back.
 #include "tc_common.cuh"
 
 namespace isopo {
@@ -67,19 +68,19 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
 
   if (kb0 < kb1) {
     if (warp == 0) {
-      if (lane == 0) {
+      if (elect_one()) {
         prefetch_tensormap(&mapG);
         int stage = 0;
         uint32_t phase = 0;
         for (long long kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdNtk)) break;
           mbar_arrive_expect_tx(full_bar(stage), stage_tx);
-          tma_load_2d(smem_base + stage * kStageBytes, &mapG, (int)(kb * kKB), 0, full_bar(stage));
+          tma_load_3d(smem_base + stage * kStageBytes, &mapG, (int)(kb & 3) * kKB, 0, (int)(kb >> 2), full_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     } else if (warp == 1) {
-      if (lane == 0) {
+      if (elect_one()) {  // elected, not "lane 0": lets the compiler keep the MMA operands in uniform registers
         const uint32_t idesc1 = make_idesc_bf16(128, n1, false, false);
         const uint32_t idesc2 = make_idesc_bf16(128, two ? n2 : 16, false, false);
         int stage = 0;
@@ -156,22 +157,24 @@ __global__ void k_mirror_upper(float* __restrict__ K, int B) {
   if (j < i) K[e] = K[(size_t)j * B + i];
 }
 
-// dW = beta dW + sum_i c_i G_i.  One thread per 16-byte chunk position of the tile-blocked store.
-__global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long chunks /* n_pad / 8 */,
+// dW = beta dW + sum_i c_i G_i.  One thread per 16-byte slot of the piece-blocked store.
+__global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long nchunks /* n_pad / 8 */,
                                                        int B, int tiles_n, int d_in, int d_out,
                                                        const float* __restrict__ coeffs, float* __restrict__ dW,
                                                        float beta) {
   __shared__ float sc[256];
   for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = coeffs[i];
   __syncthreads();
-  for (long long pos = blockIdx.x * (long long)blockDim.x + threadIdx.x; pos < chunks;
+  for (long long pos = blockIdx.x * (long long)blockDim.x + threadIdx.x; pos < nchunks;
        pos += (long long)gridDim.x * blockDim.x) {
-    const int tile = (int)(pos / (kTileElems / 8)), rem = (int)(pos % (kTileElems / 8));
-    const int j = rem / kTileM, r = rem % kTileM;
-    const int m = (tile / tiles_n) * kTileM + r, n = (tile % tiles_n) * kTileN + j * 8;
+    // pos = piece * 32 + slot in the order of one sequence; piece = (tile * 32 + j) * 4 + q
+    const long long piece = pos >> 5;
+    const int l = (int)(pos & 31), q = (int)(piece & 3), j = (int)((piece >> 2) & 31), tile = (int)(piece >> 7);
+    const int m = (tile / tiles_n) * kTileM + q * 32 + l, n = (tile % tiles_n) * kTileN + j * 8;
     if (m >= d_out || n >= d_in) continue;
     float acc[8] = {};
-    const uint4* src = G + pos;
+    const uint4* src = G + stored_slot((size_t)piece, 0, B, l);
+    const size_t chunks = 32;  // uint4 stride between successive sequences of one piece
     int i = 0;
     for (; i + 8 <= B; i += 8) {
       uint4 v[8];
@@ -216,7 +219,7 @@ isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
   CUtensorMap mapG;
   const uint32_t rows = B > 128 ? 256 : 128;
-  isopo_status s = make_map_2d_bf16(&mapG, G, (uint64_t)B, (uint64_t)L.n_pad, (uint64_t)L.n_pad, 64, rows);
+  isopo_status s = make_map_pieces_bf16(&mapG, G, (uint64_t)B, (uint64_t)(L.n_pad / kPieceElems), rows);
   if (s != ISOPO_OK) return s;
   int dev = 0, sms = 0;
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));

@@ -18,8 +18,8 @@
 // coefficient in shared memory (round to nearest even) before the MMA warp may read it, and the
 // epilogue adds float32 tiles into the row-major dW.
 //
-// Stored layout of one tile (64 KB, private to the library): element (m, n) of the tile sits at
-// ((n / 8) * 128 + m) * 8 + n % 8, so that a warp's 32 rows write 512 contiguous bytes.
+// The stored layout of G (pieces of 32 rows x 8 columns, sequence-minor) is described in
+// tc_common.cuh; one epilogue warp writes one 512-byte piece per store instruction.
 #include "tc_common.cuh"
 
 namespace isopo {
@@ -107,7 +107,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (elect_one()) {
       prefetch_tensormap(&mapY);
       prefetch_tensormap(&mapX);
       int stage = 0;
@@ -169,7 +169,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
           fence_proxy_async_smem();
         }
         __syncwarp();
-        if (lane == 0) {
+        if (elect_one()) {  // elected, not "lane 0": lets the compiler keep the operands in uniform registers
           for (int k16 = 0; k16 < n16; ++k16) {
             const uint64_t a_desc = make_sdesc_sw128(a_addr + k16 * 2048, kChunkBytes, 1024);
             const uint64_t b_desc = make_sdesc_sw128(b_addr + k16 * 2048, kChunkBytes, 1024);
@@ -181,7 +181,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
         if (++stage == kStages) { stage = 0; phase ^= 1u; }
       }
       if (!ok) break;
-      if (lane == 0) mma_commit(accfull_bar(acc));
+      if (elect_one()) mma_commit(accfull_bar(acc));
       __syncwarp();
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -197,7 +197,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTileN;
       if (!kFolded) {
-        uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)i * p.n_pad + (size_t)tile * kTileElems) + row;
+        uint4* dst = reinterpret_cast<uint4*>(p.G);
 #pragma unroll 2
         for (int jc = 0; jc < kTileN / 32; ++jc) {
           uint32_t r[32];
@@ -210,7 +210,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
             o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
             o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
             o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-            dst[(size_t)(jc * 4 + v) * kTileM] = o;
+            dst[stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane)] = o;
           }
         }
       } else {
@@ -307,6 +307,10 @@ static isopo_status sm_count(int* sms) {
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
                            const int64_t* off_dev, int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st) {
   (void)off_host;
+  // 2-CTA tiles (256 rows of G per pair) when they waste little: an odd number of 128-row tiles
+  // leaves half of the last pair idle.
+  if (L.tiles_m % 2 == 0 || L.tiles_m >= 7)
+    return bf16_seq_grad_pair(X, dY, T, d_in, d_out, off_dev, B, L, G, info, st);
   CUtensorMap mapY, mapX;
   isopo_status s = make_maps(&mapY, &mapX, X, dY, T, d_in, d_out);
   if (s != ISOPO_OK) return s;

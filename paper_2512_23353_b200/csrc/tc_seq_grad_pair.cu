@@ -1,0 +1,310 @@
+// Per-sequence weight gradients G_i = dY_i^T X_i (Alg. 1/2 reduce loop) with 2-CTA tensor-core tiles.
+//
+// Two CTAs on neighbouring SMs (a cluster of two) share one 256 x 256 tile of G_i: CTA r of the pair
+// stages dY[:, 128 columns] (its half of the tile's rows) and X[:, 128 columns] (its half of the
+// tile's columns), one thread of CTA 0 issues tcgen05.mma.cta_group::2 (256 x 256 x 16, both operands
+// token-major = "MN-major"), and each CTA ends up with its 128 x 256 half of the accumulator in its
+// own tensor memory.  A 128 x 256 tile per CTA needs 96 bytes of operands per tensor clock read from
+// shared memory and as many written by TMA, more than shared memory can move; the pair tile needs 64.
+//
+// Work units are (sequence i, pair tile), sequence-major, handed round-robin to the persistent
+// pairs, so the pairs running at one time read the same sequence's tokens out of L2.
+//
+//   warp 0          TMA producer; both CTAs' copies complete on the barrier in CTA 0
+//   warp 1, CTA 0   MMA issuer (one thread)
+//   warps 2-5       epilogue: TMEM -> registers -> bf16 (round to nearest even) -> stored gradients
+//   warp 6          zeroes the dY rows past the end of a sequence in its last slab
+//
+// Barriers.  full[s] lives in CTA 0 and counts the bytes of both CTAs; tcgen05.commit releases
+// empty[s] and raises accfull[b] in BOTH CTAs; accempty[b] in CTA 0 counts the eight epilogue warps
+// of the pair.  In the last slab of a sequence whose length is not a multiple of 16 the dY copy of
+// each CTA completes on that CTA's own tail[s] barrier instead; warp 6 waits for it, zeroes the rows
+// and arrives on fixed[s] in CTA 0, which the MMA thread waits for in addition to full[s].
+// Every wait is bounded; a CTA that gives up raises the abort flag of both CTAs, and both meet at
+// a cluster barrier before tensor memory is released.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+
+#include "tc_common.cuh"
+
+namespace isopo {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kKB = 64;                              // tokens per pipeline stage
+constexpr int kStages = 6;
+constexpr int kHalf = 128;                           // operand columns staged per CTA (both operands)
+constexpr int kChunkBytes = kKB * 128;               // one [kKB tokens][64 columns] box
+constexpr int kOperandBytes = 2 * kChunkBytes;       // this CTA's half of dY or of X for one stage
+constexpr int kStageBytes = 2 * kOperandBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+constexpr int kThreads = 224;
+constexpr uint32_t kTmemCols = 512;                  // two 256-column float32 accumulators
+constexpr int kPairN = 256;                          // columns of a pair tile (= columns of a stored tile)
+static_assert(kKB % 16 == 0 && kKB <= 256, "a stage is a whole number of 16-token MMA steps and one TMA box");
+static_assert(kSmemBytes <= 227 * 1024, "shared memory");
+
+struct PairParams {
+  const int64_t* off;
+  __nv_bfloat16* G;
+  int B, tiles_m, tiles_n;  // stored 128 x 256 tiles per gradient
+  int ptiles_m;             // pair tiles along d_out = ceil(tiles_m / 2)
+  int32_t* info;
+};
+
+// Shape of one unit's token loop, identical in every role.
+struct UnitShape {
+  int nkb;         // slabs
+  int tail_n16;    // 16-token MMA steps of the last slab
+  int tail_valid;  // token rows of the last slab that belong to the sequence
+  bool fix;        // the last step holds rows of the next sequence
+};
+__device__ __forceinline__ UnitShape unit_shape(int len) {
+  UnitShape s;
+  s.nkb = (len + kKB - 1) / kKB;
+  s.tail_valid = len - (s.nkb - 1) * kKB;
+  s.tail_n16 = (s.tail_valid + 15) >> 4;
+  s.fix = s.tail_valid < s.tail_n16 * 16;
+  return s;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapX, PairParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };                          // used in CTA 0
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };             // both CTAs
+  auto tail_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };          // both CTAs
+  auto fixed_bar = [&](int s) { return bar0 + 8u * (3 * kStages + s); };         // used in CTA 0
+  auto accfull_bar = [&](int b) { return bar0 + 8u * (4 * kStages + b); };       // both CTAs
+  auto accempty_bar = [&](int b) { return bar0 + 8u * (4 * kStages + 2 + b); };  // used in CTA 0
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 issues the MMAs
+  const uint32_t peer_abort = map_to_cta(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+      mbar_init(tail_bar(s), 1);
+      mbar_init(fixed_bar(s), 2);
+    }
+    for (int b = 0; b < 2; ++b) { mbar_init(accfull_bar(b), 1); mbar_init(accempty_bar(b), 8); }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();  // the peer's barriers exist before anything can arrive on them
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int ptiles = p.ptiles_m * p.tiles_n;
+  const long long total_units = (long long)p.B * ptiles;
+  const long long pair_id = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (elect_one()) {
+      prefetch_tensormap(&mapY);
+      prefetch_tensormap(&mapX);
+      const uint32_t full_at_leader = map_to_cta(full_bar(0), 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long u = pair_id; u < total_units && ok; u += npairs) {
+        const int i = (int)(u / ptiles), pt = (int)(u % ptiles);
+        const int ptm = pt / p.tiles_n, tn = pt % p.tiles_n;
+        const int64_t t0 = p.off[i];
+        const UnitShape us = unit_shape((int)(p.off[i + 1] - t0));
+        const int ycol = (2 * ptm + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
+        for (int kb = 0; kb < us.nkb; ++kb) {
+          if (!(ok = mbar_wait_pair(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
+          const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kOperandBytes;
+          const int y = (int)(t0 + (int64_t)kb * kKB);
+          const bool own_tail = us.fix && kb == us.nkb - 1;  // dY goes to this CTA's tail barrier
+          if (own_tail) mbar_arrive_expect_tx(tail_bar(stage), kOperandBytes);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), own_tail ? 2 * kOperandBytes : 2 * kStageBytes);
+          const uint32_t fb = full_at_leader + 8u * stage;
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            if (own_tail) tma_load_2d(a_dst + c * kChunkBytes, &mapY, ycol + c * 64, y, tail_bar(stage));
+            else tma_load_2d_pair(a_dst + c * kChunkBytes, &mapY, ycol + c * 64, y, fb);
+            tma_load_2d_pair(b_dst + c * kChunkBytes, &mapX, xcol + c * 64, y, fb);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (one thread of CTA 0)
+    // elected, not "lane 0": lets the compiler keep the MMA operands in uniform registers
+    if (rank == 0 && elect_one()) {
+      constexpr uint32_t idesc = make_idesc_bf16(256, kPairN, /*a_mn=*/true, /*b_mn=*/true);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0, fixed_phase = 0;  // fixed_phase: one bit per stage
+      bool ok = true;
+      for (long long u = pair_id; u < total_units && ok; u += npairs) {
+        const int i = (int)(u / ptiles);
+        const UnitShape us = unit_shape((int)(p.off[i + 1] - p.off[i]));
+        if (!(ok = mbar_wait_pair(accempty_bar(acc), acc_phase ^ 1u, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * kPairN;
+        for (int kb = 0; kb < us.nkb; ++kb) {
+          const bool last = kb == us.nkb - 1;
+          if (!(ok = mbar_wait_pair(full_bar(stage), phase, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
+          if (last && us.fix) {
+            // both CTAs' dY halves of this slab have landed and their stray rows are zero
+            if (!(ok = mbar_wait_pair<true>(fixed_bar(stage), (fixed_phase >> stage) & 1u, abort_flag, peer_abort, p.info,
+                                            kIdSeqGrad)))
+              break;
+            fixed_phase ^= 1u << stage;
+          }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_base + stage * kStageBytes, b_addr = a_addr + kOperandBytes;
+          const int n16 = last ? us.tail_n16 : kKB / 16;
+          for (int k16 = 0; k16 < n16; ++k16) {
+            const uint64_t a_desc = make_sdesc_sw128(a_addr + k16 * 2048, kChunkBytes, 1024);
+            const uint64_t b_desc = make_sdesc_sw128(b_addr + k16 * 2048, kChunkBytes, 1024);
+            mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | k16) != 0);
+          }
+          mma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        mma_commit_pair(accfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const uint32_t accempty_at_leader = map_to_cta(accempty_bar(0), 0);
+    uint4* dst = reinterpret_cast<uint4*>(p.G);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (long long u = pair_id; u < total_units; u += npairs) {
+      const int i = (int)(u / ptiles), pt = (int)(u % ptiles);
+      const int tm = 2 * (pt / p.tiles_n) + (int)rank, tn = pt % p.tiles_n;
+      const int tile = tm * p.tiles_n + tn;
+      if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
+      tc_fence_after_sync();
+      if (tm < p.tiles_m) {  // an odd number of row tiles leaves the last pair's second half empty
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
+#pragma unroll 2
+        for (int jc = 0; jc < kPairN / 32; ++jc) {
+          uint32_t r[32];
+          tmem_ld32(taddr + jc * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+            o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+            o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+            o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+            dst[stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane)] = o;
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(accempty_at_leader + 8u * acc);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else {
+    // ------------------------------------------------------------------ tail warp (warp 6, both CTAs)
+    // tail[s] is used only for last slabs that need the fix, so its phase is counted per stage; it
+    // cannot run ahead: the stage is not reloaded before the MMA thread has passed fixed[s].
+    const uint32_t fixed_at_leader = map_to_cta(fixed_bar(0), 0);
+    int stage = 0;
+    uint32_t tail_phase = 0;  // one bit per stage
+    for (long long u = pair_id; u < total_units; u += npairs) {
+      const int i = (int)(u / ptiles);
+      const UnitShape us = unit_shape((int)(p.off[i + 1] - p.off[i]));
+      const int ts = (stage + us.nkb - 1) % kStages;  // ring position of the last slab
+      if (us.fix) {
+        if (!mbar_wait_pair(tail_bar(ts), (tail_phase >> ts) & 1u, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
+        tail_phase ^= 1u << ts;
+        // rows [tail_valid, tail_n16*16) hold the next sequence's tokens
+        const int nbytes = (us.tail_n16 * 16 - us.tail_valid) * 128;
+        const uint32_t a_addr = smem_base + ts * kStageBytes;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const uint32_t base = a_addr + c * kChunkBytes + us.tail_valid * 128;
+          for (int o = lane * 16; o < nbytes; o += 32 * 16)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + o), "r"(0u) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(fixed_at_leader + 8u * ts);
+      }
+      stage = (ts + 1) % kStages;
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  if (*abort_flag) __nanosleep(100000);  // let TMA copies already in flight land before the CTA exits
+  tc_fence_before_sync();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still use it
+  if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+}
+
+}  // namespace
+
+isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
+                                int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st) {
+  CUtensorMap mapY, mapX;
+  isopo_status s = make_map_2d_bf16(&mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kKB);
+  if (s != ISOPO_OK) return s;
+  s = make_map_2d_bf16(&mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kKB);
+  if (s != ISOPO_OK) return s;
+  int dev = 0, sms = 0;
+  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
+  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  PairParams p{};
+  p.off = off_dev; p.G = (__nv_bfloat16*)G; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
+  p.ptiles_m = (L.tiles_m + 1) / 2;
+  p.info = info;
+  const long long units = (long long)B * p.ptiles_m * p.tiles_n;
+  // Persistent pairs with a static share of the units each: launch only as many pairs as can be
+  // resident at once (the hardware may place fewer 2-CTA clusters than there are SM pairs).
+  static int resident_pairs[64] = {};
+  if (dev < 0 || dev >= 64) return ISOPO_ERR_UNSUPPORTED;
+  if (resident_pairs[dev] == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)(sms / 2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    ISOPO_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, k_bf16_seq_grad_pair, &cfg));
+    if (n < 1) return ISOPO_ERR_UNSUPPORTED;
+    resident_pairs[dev] = std::min(n, sms / 2);
+  }
+  const int npairs = (int)std::max<long long>(1, std::min<long long>(units, resident_pairs[dev]));
+  {
+    LaunchScope scope(kIdSeqGrad, st);
+    k_bf16_seq_grad_pair<<<2 * npairs, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+}  // namespace isopo
