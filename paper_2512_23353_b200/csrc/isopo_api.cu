@@ -58,6 +58,8 @@ WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, iso
   size_t p = 0;
   L.off_offsets = p;
   p = align_up(p + sizeof(int64_t) * (size_t)(B + 1), 1024);
+  L.off_order = p;
+  p = align_up(p + sizeof(int32_t) * (size_t)B, 1024);
   L.off_tokseq = p;
   p = align_up(p + sizeof(int32_t) * (size_t)T, 1024);
   L.off_kacc = p;
@@ -192,7 +194,10 @@ isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, 
   }
   if (rp == ISOPO_PATH_GRAM) return bf16_gram(X, dY, T, d_in, d_out, tokseq, B, K, info, st);
   void* G = w + L.off_G;
-  s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, B, L, G, info, st);
+  int32_t* order = (int32_t*)(w + L.off_order);
+  s = launch_order(seq_offsets_host, B, order, st);
+  if (s != ISOPO_OK) return s;
+  s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, order, B, L, G, info, st);
   if (s != ISOPO_OK) return s;
   return bf16_ntk(G, L, B, K, info, st);
 }

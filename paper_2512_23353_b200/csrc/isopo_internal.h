@@ -57,6 +57,7 @@ class ProfilingPause {
 
 struct WsLayout {
   size_t off_offsets;  // int64 [B+1]
+  size_t off_order;    // int32 [B]       (bf16 materialised path: sequences, longest first)
   size_t off_tokseq;   // int32 [T]
   size_t off_kacc;     // float64 [B*B]   (float32 path: K accumulators)
   size_t off_G;        // stored gradients (materialised path only)
@@ -82,6 +83,8 @@ void set_cuda_error(cudaError_t e, const char* where);
 // ---- launchers (each enqueues on `st` and returns a status; none synchronises) ----
 
 isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq, cudaStream_t st);
+// order_dev[k] = index of the k-th longest sequence (B <= 256)
+isopo_status launch_order(const int64_t* off_host, int B, int32_t* order_dev, cudaStream_t st);
 
 // float32 SIMT path
 isopo_status f32_seq_grad(const float* X, const float* dY, int d_in, int d_out, const int64_t* off_dev, int B,
@@ -95,9 +98,11 @@ isopo_status f32_weight_grad(const float* X, const float* dY, int64_t T, int d_i
 
 // bf16 tcgen05 path
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
-                           const int64_t* off_dev, int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st);
+                           const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout& L, void* G,
+                           int32_t* info, cudaStream_t st);
 isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
-                                int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st);
+                                const int32_t* order_dev, int B, const WsLayout& L, void* G, int32_t* info,
+                                cudaStream_t st);
 isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t* info, cudaStream_t st);
 isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
                           float beta, cudaStream_t st);

@@ -12,6 +12,20 @@ namespace {
 constexpr int kT = 64;   // output tile edge of the SIMT GEMMs
 constexpr int kTK = 16;  // tokens staged per step
 
+// Host values travel to the device as kernel arguments (no host-to-device copy, so no hidden
+// synchronisation with the stream and nothing that reads the caller's array after the call returns).
+constexpr int kArgChunk = 384;
+struct OffsetArgs { int64_t v[kArgChunk]; };
+struct OrderArgs { int32_t v[256]; };
+__global__ void k_store_offsets(OffsetArgs a, int base, int n, int64_t* __restrict__ off) {
+  const int t = threadIdx.x;
+  if (t < n) off[base + t] = a.v[t];
+}
+__global__ void k_store_order(OrderArgs a, int n, int32_t* __restrict__ order) {
+  const int t = threadIdx.x;
+  if (t < n) order[t] = a.v[t];
+}
+
 __global__ void k_tokseq(const int64_t* __restrict__ off, int B, int64_t T, int32_t* __restrict__ tokseq) {
   for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
     int lo = 0, hi = B;  // invariant: off[lo] <= t < off[hi]
@@ -189,12 +203,31 @@ __global__ void k_f32_combine(const float* __restrict__ G, int64_t N, int B, con
 
 isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq,
                          cudaStream_t st) {
-  ISOPO_CUDA_TRY(cudaMemcpyAsync(off_dev, off_host, sizeof(int64_t) * (size_t)(B + 1), cudaMemcpyHostToDevice, st));
+  for (int base = 0; base <= B; base += kArgChunk) {
+    OffsetArgs a;
+    const int n = std::min(kArgChunk, B + 1 - base);
+    for (int t = 0; t < n; ++t) a.v[t] = off_host[base + t];
+    k_store_offsets<<<1, kArgChunk, 0, st>>>(a, base, n, off_dev);
+    ISOPO_CUDA_TRY(cudaGetLastError());
+  }
   const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
   {
     LaunchScope scope(kIdPrep, st);
     k_tokseq<<<grid, 256, 0, st>>>(off_dev, B, T, tokseq);
   }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status launch_order(const int64_t* off_host, int B, int32_t* order_dev, cudaStream_t st) {
+  if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  OrderArgs a;
+  for (int i = 0; i < B; ++i) a.v[i] = i;
+  // longest first; equal lengths keep their order
+  std::stable_sort(a.v, a.v + B, [&](int32_t x, int32_t y) {
+    return off_host[x + 1] - off_host[x] > off_host[y + 1] - off_host[y];
+  });
+  k_store_order<<<1, 256, 0, st>>>(a, B, order_dev);
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }

@@ -198,41 +198,23 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void cluster_sync_all() {  // every thread of both CTAs
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// arrival that publishes this thread's earlier shared-memory writes to the whole pair (slow: keep it
-// out of per-stage loops)
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// arrival that publishes nothing but "done" (e.g. a drained accumulator): CTA-scope release, cheap
+// Arrival on a barrier of the other CTA of the pair (CTA-scope release: it says "done", it is not a
+// cluster-wide fence, which would stall the arriving warp for hundreds of clocks).
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait inside a CTA pair.  kClusterAcquire: acquire at cluster scope, for the one case where
-// the arrival publishes the peer's ordinary shared-memory writes; completions of TMA copies and of
-// tcgen05.commit, and arrivals that only hand over tensor memory, need the CTA-scope form, which is
-// much cheaper in the MMA issuer's loop.  On giving up it also raises the peer's abort flag (`peer_abort`, a shared::cluster address) so that both
-// CTAs of the pair head for the teardown.
-template <bool kClusterAcquire = false>
+// Bounded wait inside a CTA pair: as mbar_wait, and on giving up it also raises the peer's abort
+// flag (`peer_abort`, a shared::cluster address) so that both CTAs of the pair head for the teardown.
 __device__ __forceinline__ bool mbar_wait_pair(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                uint32_t peer_abort, int32_t* info, int code) {
-  auto try_wait = [&]() { return kClusterAcquire ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
-  if (try_wait()) return true;
+  if (mbar_try_wait(bar, parity)) return true;
   const long long start = clock64();
   while (true) {
     for (int i = 0; i < 64; ++i)
-      if (try_wait()) return true;
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (clock64() - start > (1ll << 31)) {
       *abort_flag = 1;

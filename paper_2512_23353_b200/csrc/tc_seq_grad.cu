@@ -34,13 +34,16 @@ constexpr int kABytes = kTileM * kKB * 2;              // 16 KB: 2 chunks of [64
 constexpr int kBBytes = kTileN * kKB * 2;              // 32 KB: 4 chunks
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kChunkBytes = kKB * 128;                 // one [64 tokens][64 cols] box
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kMaxSeqs = 256;                          // sequences whose extents are staged in shared memory
+constexpr int kSeqInfoBytes = kMaxSeqs * 16;           // int64 first token, int32 length, int32 index
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kSeqInfoBytes;
 constexpr int kThreads = 192;
 constexpr int kThreadsFolded = 320;                    // + 4 warps that scale the dY rows
 constexpr uint32_t kTmemCols = 512;                    // two 256-column float32 accumulators
 
 struct SeqGradParams {
   const int64_t* off;
+  const int32_t* order;  // per-sequence mode: the k-th sequence to work on (longest first)
   __nv_bfloat16* G;
   int64_t n_pad;
   int B, tiles_m, tiles_n;
@@ -53,19 +56,29 @@ struct SeqGradParams {
   int nslabs, d_in, d_out;
 };
 
-// Work unit u -> (token range, tile).  Per-sequence mode: sequence-major, u = i * tiles + tile.
-// Folded mode: u = slab * tiles + tile.
+// Extents of the sequences in working order, staged in shared memory by the kernel (per-sequence mode).
+struct SeqInfo {
+  const int64_t* first;
+  const int* len;
+  const int* seq;
+};
+
+// Work unit u -> (token range, tile).  Per-sequence mode: sequence-major, u = k * tiles + tile with the
+// sequences taken longest first: round-robin over the CTAs then gives every CTA a regular sample of
+// the sorted lengths, i.e. nearly the same number of tokens.  Folded mode: u = slab * tiles + tile.
 template <bool kFolded>
-__device__ __forceinline__ void decode_unit(const SeqGradParams& p, long long u, int tiles, int& tile, int64_t& t0,
-                                            int64_t& t1, int& seq) {
-  seq = (int)(u / tiles);
+__device__ __forceinline__ void decode_unit(const SeqGradParams& p, const SeqInfo& si, long long u, int tiles, int& tile,
+                                            int64_t& t0, int64_t& t1, int& seq) {
+  const int k = (int)(u / tiles);
   tile = (int)(u % tiles);
   if (kFolded) {
-    t0 = (int64_t)seq * p.slab;
+    seq = k;
+    t0 = (int64_t)k * p.slab;
     t1 = min(p.T, t0 + p.slab);
   } else {
-    t0 = p.off[seq];
-    t1 = p.off[seq + 1];
+    seq = si.seq[k];
+    t0 = si.first[k];
+    t1 = t0 + si.len[k];
   }
 }
 
@@ -84,6 +97,21 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
   auto scaled_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 4 + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kStages + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // read once: the roles look the extents up at every unit, and a global load there would stall
+  // the MMA warp for longer than its queue of MMAs lasts
+  int64_t* s_first = reinterpret_cast<int64_t*>(smem + kStages * kStageBytes + 256);
+  int* s_len = reinterpret_cast<int*>(s_first + kMaxSeqs);
+  int* s_seq = s_len + kMaxSeqs;
+  if (!kFolded) {
+    for (int k = threadIdx.x; k < p.B; k += blockDim.x) {
+      const int i = p.order[k];
+      const int64_t t0 = p.off[i];
+      s_first[k] = t0;
+      s_len[k] = (int)(p.off[i + 1] - t0);
+      s_seq[k] = i;
+    }
+  }
+  const SeqInfo si{s_first, s_len, s_seq};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -116,7 +144,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
       for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
         int i, tile;
         int64_t t0, t1;
-        decode_unit<kFolded>(p, u, tiles_per_seq, tile, t0, t1, i);
+        decode_unit<kFolded>(p, si, u, tiles_per_seq, tile, t0, t1, i);
         const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
         const int nkb = (int)((t1 - t0 + kKB - 1) / kKB);
         for (int kb = 0; kb < nkb; ++kb) {
@@ -143,7 +171,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
     for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
       int i, tile;
       int64_t t0, t1;
-      decode_unit<kFolded>(p, u, tiles_per_seq, tile, t0, t1, i);
+      decode_unit<kFolded>(p, si, u, tiles_per_seq, tile, t0, t1, i);
       const int len = (int)(t1 - t0);
       const int nkb = (len + kKB - 1) / kKB;
       if (!(ok = mbar_wait(accempty_bar(acc), acc_phase ^ 1u, abort_flag, p.info, kIdSeqGrad))) break;
@@ -192,7 +220,8 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
     int acc = 0;
     uint32_t acc_phase = 0;
     for (long long u = blockIdx.x; u < total_units; u += gridDim.x) {
-      const int i = (int)(u / tiles_per_seq), tile = (int)(u % tiles_per_seq);
+      const int tile = (int)(u % tiles_per_seq);
+      const int i = kFolded ? 0 : si.seq[u / tiles_per_seq];
       if (!mbar_wait(accfull_bar(acc), acc_phase, abort_flag, p.info, kIdSeqGrad)) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTileN;
@@ -252,7 +281,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
     for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
       int i, tile;
       int64_t t0, t1;
-      decode_unit<kFolded>(p, u, tiles_per_seq, tile, t0, t1, i);
+      decode_unit<kFolded>(p, si, u, tiles_per_seq, tile, t0, t1, i);
       const int nkb = (int)((t1 - t0 + kKB - 1) / kKB);
       for (int kb = 0; kb < nkb; ++kb) {
         const int64_t t = t0 + (int64_t)kb * kKB + r;
@@ -305,12 +334,13 @@ static isopo_status sm_count(int* sms) {
 }
 
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
-                           const int64_t* off_dev, int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st) {
+                           const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout& L, void* G,
+                           int32_t* info, cudaStream_t st) {
   (void)off_host;
   // 2-CTA tiles (256 rows of G per pair) when they waste little: an odd number of 128-row tiles
   // leaves half of the last pair idle.
   if (L.tiles_m % 2 == 0 || L.tiles_m >= 7)
-    return bf16_seq_grad_pair(X, dY, T, d_in, d_out, off_dev, B, L, G, info, st);
+    return bf16_seq_grad_pair(X, dY, T, d_in, d_out, off_dev, order_dev, B, L, G, info, st);
   CUtensorMap mapY, mapX;
   isopo_status s = make_maps(&mapY, &mapX, X, dY, T, d_in, d_out);
   if (s != ISOPO_OK) return s;
@@ -318,7 +348,7 @@ isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, i
   if ((s = sm_count(&sms)) != ISOPO_OK) return s;
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   SeqGradParams p{};
-  p.off = off_dev; p.G = (__nv_bfloat16*)G; p.n_pad = L.n_pad; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
+  p.off = off_dev; p.order = order_dev; p.G = (__nv_bfloat16*)G; p.n_pad = L.n_pad; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
   p.info = info;
   const long long units = (long long)B * L.tiles_m * L.tiles_n;
   const int grid = (int)std::min<long long>(units, sms);

@@ -7,8 +7,10 @@
 // own tensor memory.  A 128 x 256 tile per CTA needs 96 bytes of operands per tensor clock read from
 // shared memory and as many written by TMA, more than shared memory can move; the pair tile needs 64.
 //
-// Work units are (sequence i, pair tile), sequence-major, handed round-robin to the persistent
-// pairs, so the pairs running at one time read the same sequence's tokens out of L2.
+// Work units are (sequence, pair tile), sequence-major with the sequences taken longest first, handed
+// round-robin to the persistent pairs: the pairs running at one time read the same sequence's tokens
+// out of L2, and every pair gets a regular sample of the sorted lengths, i.e. nearly the same number
+// of tokens.
 //
 //   warp 0          TMA producer; both CTAs' copies complete on the barrier in CTA 0
 //   warp 1, CTA 0   MMA issuer (one thread)
@@ -40,7 +42,9 @@ constexpr int kHalf = 128;                           // operand columns staged p
 constexpr int kChunkBytes = kKB * 128;               // one [kKB tokens][64 columns] box
 constexpr int kOperandBytes = 2 * kChunkBytes;       // this CTA's half of dY or of X for one stage
 constexpr int kStageBytes = 2 * kOperandBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+constexpr int kMaxSeqs = 256;                        // sequences whose extents are staged in shared memory
+constexpr int kSeqInfoBytes = kMaxSeqs * 16;         // int64 first token, int32 length, int32 index
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/ + kSeqInfoBytes;
 constexpr int kThreads = 224;
 constexpr uint32_t kTmemCols = 512;                  // two 256-column float32 accumulators
 constexpr int kPairN = 256;                          // columns of a pair tile (= columns of a stored tile)
@@ -49,6 +53,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory");
 
 struct PairParams {
   const int64_t* off;
+  const int32_t* order;     // the k-th sequence to work on (longest first)
   __nv_bfloat16* G;
   int B, tiles_m, tiles_n;  // stored 128 x 256 tiles per gradient
   int ptiles_m;             // pair tiles along d_out = ceil(tiles_m / 2)
@@ -86,6 +91,18 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
   auto accempty_bar = [&](int b) { return bar0 + 8u * (4 * kStages + 2 + b); };  // used in CTA 0
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * kStages + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // extents of the sequences in working order, read once: the roles look them up at every unit,
+  // and a global load there would stall the MMA thread for longer than its queue of MMAs lasts
+  int64_t* s_first = reinterpret_cast<int64_t*>(smem + kStages * kStageBytes + 512);
+  int* s_len = reinterpret_cast<int*>(s_first + kMaxSeqs);
+  int* s_seq = s_len + kMaxSeqs;
+  for (int k = threadIdx.x; k < p.B; k += kThreads) {
+    const int i = p.order[k];
+    const int64_t t0 = p.off[i];
+    s_first[k] = t0;
+    s_len[k] = (int)(p.off[i + 1] - t0);
+    s_seq[k] = i;
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();  // 0 issues the MMAs
@@ -123,10 +140,10 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
       uint32_t phase = 0;
       bool ok = true;
       for (long long u = pair_id; u < total_units && ok; u += npairs) {
-        const int i = (int)(u / ptiles), pt = (int)(u % ptiles);
+        const int k = (int)(u / ptiles), pt = (int)(u % ptiles);
         const int ptm = pt / p.tiles_n, tn = pt % p.tiles_n;
-        const int64_t t0 = p.off[i];
-        const UnitShape us = unit_shape((int)(p.off[i + 1] - t0));
+        const int64_t t0 = s_first[k];
+        const UnitShape us = unit_shape(s_len[k]);
         const int ycol = (2 * ptm + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
         for (int kb = 0; kb < us.nkb; ++kb) {
           if (!(ok = mbar_wait_pair(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
@@ -155,8 +172,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
       uint32_t phase = 0, acc_phase = 0, fixed_phase = 0;  // fixed_phase: one bit per stage
       bool ok = true;
       for (long long u = pair_id; u < total_units && ok; u += npairs) {
-        const int i = (int)(u / ptiles);
-        const UnitShape us = unit_shape((int)(p.off[i + 1] - p.off[i]));
+        const UnitShape us = unit_shape(s_len[u / ptiles]);
         if (!(ok = mbar_wait_pair(accempty_bar(acc), acc_phase ^ 1u, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * kPairN;
         for (int kb = 0; kb < us.nkb; ++kb) {
@@ -164,8 +180,8 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
           if (!(ok = mbar_wait_pair(full_bar(stage), phase, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
           if (last && us.fix) {
             // both CTAs' dY halves of this slab have landed and their stray rows are zero
-            if (!(ok = mbar_wait_pair<true>(fixed_bar(stage), (fixed_phase >> stage) & 1u, abort_flag, peer_abort, p.info,
-                                            kIdSeqGrad)))
+            if (!(ok = mbar_wait_pair(fixed_bar(stage), (fixed_phase >> stage) & 1u, abort_flag, peer_abort, p.info,
+                                      kIdSeqGrad)))
               break;
             fixed_phase ^= 1u << stage;
           }
@@ -193,7 +209,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
     int acc = 0;
     uint32_t acc_phase = 0;
     for (long long u = pair_id; u < total_units; u += npairs) {
-      const int i = (int)(u / ptiles), pt = (int)(u % ptiles);
+      const int i = s_seq[u / ptiles], pt = (int)(u % ptiles);
       const int tm = 2 * (pt / p.tiles_n) + (int)rank, tn = pt % p.tiles_n;
       const int tile = tm * p.tiles_n + tn;
       if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
@@ -229,8 +245,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
     int stage = 0;
     uint32_t tail_phase = 0;  // one bit per stage
     for (long long u = pair_id; u < total_units; u += npairs) {
-      const int i = (int)(u / ptiles);
-      const UnitShape us = unit_shape((int)(p.off[i + 1] - p.off[i]));
+      const UnitShape us = unit_shape(s_len[u / ptiles]);
       const int ts = (stage + us.nkb - 1) % kStages;  // ring position of the last slab
       if (us.fix) {
         if (!mbar_wait_pair(tail_bar(ts), (tail_phase >> ts) & 1u, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
@@ -246,7 +261,10 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(fixed_at_leader + 8u * ts);
+        // The stores above were performed in this CTA's shared memory before the proxy fence
+        // returned, and only this CTA's tensor core reads them; the arrival merely tells the MMA
+        // thread so.  A cluster-scope release here costs the MMA thread ~1500 clocks per unit.
+        if (lane == 0) mbar_arrive_remote(fixed_at_leader + 8u * ts);
       }
       stage = (ts + 1) % kStages;
     }
@@ -264,7 +282,8 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
 }  // namespace
 
 isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
-                                int B, const WsLayout& L, void* G, int32_t* info, cudaStream_t st) {
+                                const int32_t* order_dev, int B, const WsLayout& L, void* G, int32_t* info,
+                                cudaStream_t st) {
   CUtensorMap mapY, mapX;
   isopo_status s = make_map_2d_bf16(&mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kKB);
   if (s != ISOPO_OK) return s;
@@ -275,7 +294,7 @@ isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   PairParams p{};
-  p.off = off_dev; p.G = (__nv_bfloat16*)G; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
+  p.off = off_dev; p.order = order_dev; p.G = (__nv_bfloat16*)G; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
   p.ptiles_m = (L.tiles_m + 1) / 2;
   p.info = info;
   const long long units = (long long)B * p.ptiles_m * p.tiles_n;

@@ -128,3 +128,25 @@ def test_small_llm_config_sampled(b):
         assert rel_fro(res.K.cpu().numpy(), K_o) <= TOL
         assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL
         assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_ragged_tails_many_short_sequences(b, seed):
+    """200 sequences of 1..130 tokens on a layer shape that takes the 2-CTA kernel: almost every
+    sequence ends inside a 16-token MMA step, several sequences share one 64-token slab, and the
+    slabs of successive sequences chase each other through the ring.  A token row of the next
+    sequence leaking into G_i would change K_ii by O(1/L_i), far above the tolerance."""
+    rng = np.random.default_rng(1234 + seed)
+    Ls = rng.integers(1, 131, size=200).tolist()
+    X, dY, off, A = _inputs(Ls, 256, 256, 700 + seed)
+    G = orc.sequence_gradients(to_f64(X), to_f64(dY), off)
+    K_o = orc.ntk(G)
+    res = b.isopo_layer(X, dY, off, A, b.VAR_NORMALISED, 0.0, b.PATH_MATERIALISE)
+    assert res.info == 0
+    K = res.K.cpu().numpy()
+    assert rel_fro(K, K_o) <= TOL
+    # every diagonal entry on its own (a leak into one short sequence would drown in the Frobenius norm)
+    d, d_o = np.diag(K), np.diag(K_o)
+    assert np.max(np.abs(d - d_o) / d_o) <= TOL
+    c_o = orc.transform_advantages(K_o, to_f64(A), orc.NORMALISED, 0.0)
+    assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
