@@ -28,6 +28,9 @@ next to the function it affects):
     `scaling * grad`); regularisation terms are absolute numbers supplied by
     the caller; no 1/n, 1/B or 1/T factor appears anywhere.
 
+The token-sampled Fisher-norm estimator of Algorithm 1 (`sampled_fisher_norm_sq`) takes the sampled
+row indices as an input; the K-only estimator above is the same formula with whole sequences as samples.
+
 Pin status: every function below is pinned by closed forms, brute force and
 invariants in tests/test_oracle_pins.py (the paper prints no numeric example).
 """
@@ -91,6 +94,42 @@ def fisher_norm_sq(K, normalise=True):
     if normalise:
         return F2 / np.trace(K)
     return F2 / B
+
+
+def sampled_fisher_norm_sq(X, dY, off, sample_rows):
+    """Squared Fisher norm of every sequence gradient as Algorithm 1 estimates it, from
+    `n_overlap_samples` token rows (`sample_rows`, drawn by the caller: the listing's `randperm`).
+
+    a0 = act_in[samples], g0 = g_out[samples]; per sequence, with G_i = grad_out.T @ act_in,
+        F_norm = ||sum((g0 @ G_i) * a0, dim=1)|| / || ||g0_j|| * ||a0_j|| ||
+    i.e. the last display of "Efficient implementation" (Eq. one over Eq. two).  Returns F_norm^2, [B].
+    """
+    X, dY = _f64(X), _f64(dY)
+    off = np.asarray(off, dtype=np.int64)
+    rows = np.asarray(sample_rows, dtype=np.int64)
+    a0 = X[rows]
+    g0 = dY[rows]
+    denom = np.linalg.norm(np.linalg.norm(g0, axis=1) * np.linalg.norm(a0, axis=1))
+    B = off.shape[0] - 1
+    F2 = np.empty(B, dtype=np.float64)
+    for i in range(B):
+        seq = slice(int(off[i]), int(off[i + 1]))
+        seq_logprob_grad = dY[seq].T @ X[seq]
+        F_norm = np.linalg.norm(np.sum((g0 @ seq_logprob_grad) * a0, axis=1)) / denom
+        F2[i] = F_norm ** 2
+    return F2
+
+
+def sampled_coefficients(F2, A, lam=0.0):
+    """Algorithm 1's re-scaling: c_i = A_i / sqrt(F_norm_i^2 + regularization)."""
+    return _f64(A) / np.sqrt(_f64(F2) + lam)
+
+
+def isopo_layer_sampled(X, dY, off, A, sample_rows, lam=0.0):
+    """Algorithm 1 as printed: (X, dY, partition, A, sampled rows) -> (F_norm^2, c, dW)."""
+    F2 = sampled_fisher_norm_sq(X, dY, off, sample_rows)
+    c = sampled_coefficients(F2, A, lam)
+    return F2, c, weight_gradient(sequence_gradients(X, dY, off), c)
 
 
 def transform_advantages(K, A, variant, lam=0.0, pqr=None, regs=None):

@@ -308,6 +308,73 @@ def test_weight_gradient_special_cases():
 
 # ----------------------------------------------------------------------------- planted mistakes are caught
 
+# ----------------------------------------------------------------------------- Algorithm 1's sampled estimator
+def _sampled_bruteforce(X, dY, off, rows):
+    """Eq. (formal-F-norm) from its words: sum_j (v . g^(j))^2 / sum_j ||g^(j)||^2 with v = G_i as an
+    explicit matrix (four-loop brute force) and every g^(j) = g_out_j a_in_j^T built as an explicit matrix."""
+    G = _G_bruteforce(X, dY, off)
+    gs = [np.outer(dY[j], X[j]) for j in rows]
+    den = sum(float(np.sum(g * g)) for g in gs)
+    return np.array([sum(float(np.sum(G[i] * g)) ** 2 for g in gs) / den for i in range(len(off) - 1)])
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_sampled_estimator_equals_explicit_rank_one_sum(seed):
+    X, dY, off, _ = _problem(40 + seed)
+    rng = np.random.default_rng(seed)
+    rows = rng.permutation(int(off[-1]))[: max(1, int(off[-1]) // 2)]
+    np.testing.assert_allclose(orc.sampled_fisher_norm_sq(X, dY, off, rows), _sampled_bruteforce(X, dY, off, rows),
+                               rtol=1e-11)
+
+
+def test_sampled_estimator_hand_example():
+    # one sequence of two tokens, 1 x 1 layer: G = 2*3 + (-1)*4 = 2; sample = token 1: g0 = -1, a0 = 4
+    # numerator (g0 * G * a0)^2 = (-8)^2 = 64, denominator (|g0| |a0|)^2 = 16  ->  F^2 = 4 = G^2
+    X = np.array([[3.0], [4.0]])
+    dY = np.array([[2.0], [-1.0]])
+    F2 = orc.sampled_fisher_norm_sq(X, dY, [0, 2], [1])
+    np.testing.assert_allclose(F2, [4.0], rtol=1e-14)
+    np.testing.assert_allclose(orc.sampled_coefficients(F2, [3.0], lam=5.0), [1.0], rtol=1e-14)  # 3 / sqrt(4 + 5)
+
+
+def test_sampled_estimator_with_all_tokens_of_single_token_sequences_is_the_K_only_estimator():
+    """If every sequence is one token and every token is sampled, the position-wise samples ARE the
+    sequence gradients, so Algorithm 1's estimate must equal sum_j K_ij^2 / sum_j K_jj."""
+    rng = np.random.default_rng(5)
+    T = 9
+    X, dY = rng.standard_normal((T, 5)), rng.standard_normal((T, 3))
+    off = np.arange(T + 1)
+    K = (dY @ dY.T) * (X @ X.T)  # closed form for single-token sequences
+    want = np.sum(K * K, axis=1) / np.trace(K)
+    np.testing.assert_allclose(orc.sampled_fisher_norm_sq(X, dY, off, np.arange(T)), want, rtol=1e-11)
+    np.testing.assert_allclose(orc.fisher_norm_sq(K), want, rtol=1e-12)
+
+
+def test_sampled_estimator_invariances_and_bound():
+    X, dY, off, A = _problem(77, B=6)
+    T = int(off[-1])
+    rows = np.array([0, T - 1, T // 2, 1])
+    F2 = orc.sampled_fisher_norm_sq(X, dY, off, rows)
+    # order of the samples does not matter; a repeated sample set gives the same ratio
+    np.testing.assert_allclose(orc.sampled_fisher_norm_sq(X, dY, off, rows[::-1]), F2, rtol=1e-12)
+    np.testing.assert_allclose(orc.sampled_fisher_norm_sq(X, dY, off, np.concatenate([rows, rows])), F2, rtol=1e-12)
+    # Cauchy-Schwarz: (G . g^(j))^2 <= ||G||^2 ||g^(j)||^2, hence F_i^2 <= ||G_i||^2 = K_ii
+    K = orc.ntk(orc.sequence_gradients(X, dY, off))
+    assert np.all(F2 <= np.diag(K) * (1 + 1e-12))
+    # scaling the back-propagated gradients by s scales G_i by s and every sample by s: F^2 scales by s^2
+    np.testing.assert_allclose(orc.sampled_fisher_norm_sq(X, 3.0 * dY, off, rows), 9.0 * F2, rtol=1e-12)
+    # a sample orthogonal to a sequence's gradient contributes nothing to it: d_in-disjoint supports
+    Xo, dYo = np.zeros((4, 4)), np.ones((4, 2))
+    Xo[0, 0] = Xo[1, 1] = 1.0   # sequence 0 lives on input coordinates 0, 1
+    Xo[2, 2] = Xo[3, 3] = 1.0   # sequence 1 on 2, 3
+    F2o = orc.sampled_fisher_norm_sq(Xo, dYo, [0, 2, 4], [0])   # the only sample is a token of sequence 0
+    assert F2o[1] == 0.0 and F2o[0] > 0.0
+    # the whole Algorithm-1 layer: dW = sum_i A_i / sqrt(F_i^2 + reg) G_i
+    F2b, c, dW = orc.isopo_layer_sampled(X, dY, off, A, rows, lam=0.3)
+    G = _G_bruteforce(X, dY, off)
+    np.testing.assert_allclose(dW, sum(A[i] / np.sqrt(F2[i] + 0.3) * G[i] for i in range(6)), rtol=1e-11)
+
+
 def test_pins_catch_planted_mistakes(monkeypatch):
     """Each mistake planted in the oracle (an off-by-one partition, a one-sided kernel fill, a
     dropped normalisation, a wrong regulariser sign) makes a pin above fail."""
@@ -328,7 +395,18 @@ def test_pins_catch_planted_mistakes(monkeypatch):
     def transform_wrong_sign(K, A, variant, lam=0.0, pqr=None, regs=None):
         return true_tr(K, A, variant, -lam, pqr, regs)
 
+    true_sampled = orc.sampled_fisher_norm_sq
+
+    def sampled_missing_normalisation(X, dY, off, rows):   # drops the division by sum_j ||g^(j)||^2
+        Xs, dYs = np.asarray(X, float)[np.asarray(rows)], np.asarray(dY, float)[np.asarray(rows)]
+        return true_sampled(X, dY, off, rows) * np.sum(np.sum(dYs * dYs, 1) * np.sum(Xs * Xs, 1))
+
+    def sampled_transposed_samples(X, dY, off, rows):      # takes the samples' rows from the wrong end
+        return true_sampled(X, dY, off, (int(np.asarray(off)[-1]) - 1) - np.asarray(rows))
+
     plants = [
+        ("sampled_fisher_norm_sq", sampled_missing_normalisation, test_sampled_estimator_hand_example),
+        ("sampled_fisher_norm_sq", sampled_transposed_samples, lambda: test_sampled_estimator_equals_explicit_rank_one_sum(1)),
         ("sequence_gradients", seq_off_by_one, lambda: test_G_matches_four_loop_bruteforce_and_Kii_is_its_norm(0)),
         ("ntk", ntk_one_sided, lambda: test_K_equals_rank_one_route(3)),
         ("fisher_norm_sq", f2_unnormalised, lambda: test_normalised_variant_gives_unit_fisher_norm(11)),
