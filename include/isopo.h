@@ -159,6 +159,38 @@ ISOPO_API isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dt
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_sampled_coefficients: the non-interacting update as Algorithm 1 prints it, with the Fisher
+ * norm of every sequence gradient estimated from sampled token positions (Sec. 2.2, "Estimating the
+ * Fisher metric" and "Efficient implementation") instead of from K.
+ *
+ * With a0 = X[sample_rows], g0 = dY[sample_rows] (Algorithm 1's `overlap_samples`; the caller draws
+ * them, e.g. the first n of a random permutation of the T token rows):
+ *     F_i^2 = sum_j (g0_j . G_i a0_j)^2 / sum_j (||g0_j|| ||a0_j||)^2        (Eq. one over Eq. two)
+ *     coeffs[i] = A_i / sqrt(F_i^2 + lambda)                                  (`rescaling`)
+ * G_i is never formed: g0_j . G_i a0_j = sum_{t in i} (g0_j . dY_t)(a0_j . x_t), so tiles of
+ * a0 X^T and g0 dY^T are formed in tensor memory, multiplied elementwise and summed per sequence,
+ * at about n_samples (d_in + d_out) / (d_in d_out) of the cost of the weight-gradient GEMM.
+ * Follow it with isopo_weight_grad(..., ISOPO_PATH_GRAM, ...) for dW = sum_i coeffs[i] G_i; a
+ * workspace of isopo_sampled_workspace_bytes() bytes serves that call too.
+ *
+ *   sample_rows_host  host, int64 [n_samples], each in [0, T); read before the call returns
+ *   n_samples         1 .. ISOPO_MAX_SAMPLES
+ *   A                 dev, float32 [B]
+ *   lambda            absolute regulariser, >= 0
+ *   coeffs            dev, float32 [B], overwritten
+ *   F2                dev, float32 [B] or NULL: the estimates F_i^2 themselves
+ *   ws, ws_bytes      dev workspace of isopo_sampled_workspace_bytes(...) bytes, 1024-byte aligned
+ * Other arguments and conventions as for isopo_layer_gram.
+ */
+#define ISOPO_MAX_SAMPLES 4096
+ISOPO_API size_t isopo_sampled_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, int n_samples);
+ISOPO_API isopo_status isopo_sampled_coefficients(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in,
+                                                  int d_out, const int64_t* seq_offsets_host, int B,
+                                                  const int64_t* sample_rows_host, int n_samples, const float* A,
+                                                  float lambda, float* coeffs, float* F2, void* ws, size_t ws_bytes,
+                                                  int32_t* info, void* cuda_stream);
+
+/*
  * isopo_layer_gram_static: isopo_layer_gram on the GRAM route without a caller workspace and
  * without any allocation (the paper has no counterpart; this exists for the way the library gets
  * embedded).
@@ -197,7 +229,7 @@ ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, is
  * (host, ISOPO_NUM_KERNELS entries each, overwritten) and forgets them.  Launch counts are kept
  * even while event timing is disabled.  Not thread-safe; meant for benchmarks.
  */
-#define ISOPO_NUM_KERNELS 13
+#define ISOPO_NUM_KERNELS 15
 ISOPO_API void isopo_profile_enable(int on);
 ISOPO_API isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_kernel);
 ISOPO_API const char* isopo_kernel_name(int kernel_id);

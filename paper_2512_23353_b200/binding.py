@@ -27,9 +27,11 @@ EXPORTS = (
     "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",
     "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad",
     "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
+    "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
 )
+MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
-NUM_KERNELS = 13
+NUM_KERNELS = 15
 
 
 class IsopoError(RuntimeError):
@@ -66,6 +68,12 @@ def _load():
     lib.isopo_layer_gram_static.restype = c.c_int
     lib.isopo_layer_gram_static.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
                                             c.c_int, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.isopo_sampled_workspace_bytes.restype = c.c_size_t
+    lib.isopo_sampled_workspace_bytes.argtypes = [c.c_int, c.c_int64, c.c_int, c.c_int, c.c_int, c.c_int]
+    lib.isopo_sampled_coefficients.restype = c.c_int
+    lib.isopo_sampled_coefficients.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
+                                               c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_float, c.c_void_p,
+                                               c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
     lib.isopo_profile_enable.restype = None
     lib.isopo_profile_enable.argtypes = [c.c_int]
     lib.isopo_profile_collect.restype = c.c_int
@@ -177,6 +185,35 @@ def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, s
                                coeffs.data_ptr(), off.ctypes.data, B, path, dW.data_ptr(), float(beta),
                                ws.data_ptr(), ws.numel(), info.data_ptr(), _stream())
     _check(st, "isopo_weight_grad")
+
+
+def isopo_sampled_workspace_bytes(dtype: int, T: int, d_in: int, d_out: int, B: int, n_samples: int) -> int:
+    return lib.isopo_sampled_workspace_bytes(dtype, T, d_in, d_out, B, n_samples)
+
+
+def alloc_sampled_workspace(dtype: int, T: int, d_in: int, d_out: int, B: int, n_samples: int, device="cuda"):
+    n = isopo_sampled_workspace_bytes(dtype, T, d_in, d_out, B, n_samples)
+    if n == 0:
+        raise IsopoError(ERR_INVALID_ARG, "isopo_sampled_workspace_bytes: invalid sizes")
+    raw = torch.empty(n + 1024, dtype=torch.uint8, device=device)
+    shift = (-raw.data_ptr()) % 1024
+    return raw[shift:shift + n]
+
+
+def isopo_sampled_coefficients(X: torch.Tensor, dY: torch.Tensor, seq_offsets, sample_rows, A: torch.Tensor, lam: float,
+                               coeffs: torch.Tensor, ws: torch.Tensor, info: torch.Tensor, F2: torch.Tensor = None) -> None:
+    """Algorithm 1's coefficients from sampled token rows (the caller draws `sample_rows`)."""
+    off = _offsets(seq_offsets)
+    B = off.shape[0] - 1
+    rows = np.ascontiguousarray(np.asarray(sample_rows, dtype=np.int64))
+    assert rows.ndim == 1 and X.is_cuda and dY.is_cuda and X.is_contiguous() and dY.is_contiguous() and X.dtype == dY.dtype
+    assert A.dtype == torch.float32 and coeffs.dtype == torch.float32 and A.numel() == B and coeffs.numel() == B
+    assert F2 is None or (F2.dtype == torch.float32 and F2.numel() == B)
+    st = lib.isopo_sampled_coefficients(X.data_ptr(), dY.data_ptr(), _dtype_code(X), X.shape[0], X.shape[1], dY.shape[1],
+                                        off.ctypes.data, B, rows.ctypes.data, rows.shape[0], A.data_ptr(), float(lam),
+                                        coeffs.data_ptr(), F2.data_ptr() if F2 is not None else None, ws.data_ptr(),
+                                        ws.numel(), info.data_ptr(), _stream())
+    _check(st, "isopo_sampled_coefficients")
 
 
 def isopo_profile_enable(on: bool) -> None:

@@ -145,7 +145,8 @@ isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_ke
 const char* isopo_kernel_name(int id) {
   static const char* names[kIdCount] = {"k_tokseq", "k_bf16_seq_grad", "k_bf16_ntk", "k_bf16_gram", "k_bf16_weight_grad",
                                         "k_bf16_combine", "k_transform", "k_mirror_upper", "k_f32_seq_grad",
-                                        "k_f32_ntk", "k_f32_gram", "k_f32_weight_grad", "k_f32_combine"};
+                                        "k_f32_ntk", "k_f32_gram", "k_f32_weight_grad", "k_f32_combine",
+                                        "k_sampled", "k_sampled_aux"};
   return id >= 0 && id < kIdCount ? names[id] : "unknown";
 }
 
@@ -200,6 +201,34 @@ isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, 
   s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, order, B, L, G, info, st);
   if (s != ISOPO_OK) return s;
   return bf16_ntk(G, L, B, K, info, st);
+}
+
+size_t isopo_sampled_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, int n_samples) {
+  if (!sizes_ok(dtype, T, d_in, d_out, B) || n_samples < 1 || n_samples > ISOPO_MAX_SAMPLES) return 0;
+  return sampled_layout(dtype, T, d_in, d_out, B, n_samples).total;
+}
+
+isopo_status isopo_sampled_coefficients(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                                        const int64_t* seq_offsets_host, int B, const int64_t* sample_rows_host,
+                                        int n_samples, const float* A, float lambda, float* coeffs, float* F2, void* ws,
+                                        size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  if (!A || !coeffs || !info || !sample_rows_host) return ISOPO_ERR_INVALID_ARG;
+  if (!(lambda >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
+  isopo_status s = check_layer_args(X, dY, dtype, T, d_in, d_out, seq_offsets_host, B, ISOPO_PATH_GRAM, ws);
+  if (s != ISOPO_OK) return s;
+  if (n_samples < 1 || n_samples > ISOPO_MAX_SAMPLES) return ISOPO_ERR_INVALID_ARG;
+  for (int j = 0; j < n_samples; ++j)
+    if (sample_rows_host[j] < 0 || sample_rows_host[j] >= T) return ISOPO_ERR_INVALID_ARG;
+  const SampledLayout S = sampled_layout(dtype, T, d_in, d_out, B, n_samples);
+  if (ws_bytes < S.total) return ISOPO_ERR_WORKSPACE;
+  const WsLayout L = ws_layout(dtype, T, d_in, d_out, B, ISOPO_PATH_GRAM);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* w = (char*)ws;
+  int32_t* tokseq = (int32_t*)(w + L.off_tokseq);
+  s = launch_prep(seq_offsets_host, B, T, (int64_t*)(w + L.off_offsets), tokseq, st);
+  if (s != ISOPO_OK) return s;
+  return sampled_coefficients(X, dY, dtype, T, d_in, d_out, tokseq, B, sample_rows_host, n_samples, w, S, A, lambda, coeffs,
+                              F2, info, st);
 }
 
 isopo_status isopo_transform_advantages(const float* K, const float* A, int B, isopo_variant variant, float lambda,

@@ -30,7 +30,9 @@ enum KernelId : int {
   kIdF32Gram = 10,
   kIdF32WeightGrad = 11,
   kIdF32Combine = 12,
-  kIdCount = 13
+  kIdSampled = 13,     // M^T of the token-sampled estimator (tensor-core or float32 kernel)
+  kIdSampledAux = 14,  // its gather and finishing kernels
+  kIdCount = 15
 };
 
 // Brackets one kernel launch with CUDA events while profiling is enabled (isopo_profile_enable);
@@ -70,6 +72,13 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path resolved);
 
+// Workspace of isopo_sampled_coefficients: the Gram-route prefix (offsets, order, token map), then
+// the sampled row indices, the gathered rows a0 / g0, M^T and the denominator.
+struct SampledLayout {
+  size_t off_rows, off_a0, off_g0, off_mt, off_den, total;
+};
+SampledLayout sampled_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, int n_samples);
+
 void set_cuda_error(cudaError_t e, const char* where);
 #define ISOPO_CUDA_TRY(expr)                                  \
   do {                                                        \
@@ -83,6 +92,8 @@ void set_cuda_error(cudaError_t e, const char* where);
 // ---- launchers (each enqueues on `st` and returns a status; none synchronises) ----
 
 isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq, cudaStream_t st);
+// n host values -> device array, passed as kernel arguments (no host-to-device copy)
+isopo_status store_i64(const int64_t* host, int64_t n, int64_t* dev, cudaStream_t st);
 // order_dev[k] = index of the k-th longest sequence (B <= 256)
 isopo_status launch_order(const int64_t* off_host, int B, int32_t* order_dev, cudaStream_t st);
 
@@ -110,6 +121,14 @@ isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d
                        float* K, int32_t* info, cudaStream_t st);
 isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* coeffs,
                               const int32_t* tokseq, float* dW, float beta, int32_t* info, cudaStream_t st);
+
+// token-sampled estimator of Algorithm 1
+isopo_status bf16_sampled(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
+                          const void* A0, const void* G0, int n_samples, float* Mt, int32_t* info, cudaStream_t st);
+isopo_status sampled_coefficients(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
+                                  const int32_t* tokseq, int B, const int64_t* rows_host, int n_samples, char* ws,
+                                  const SampledLayout& S, const float* A, float lambda, float* coeffs, float* F2,
+                                  int32_t* info, cudaStream_t st);
 
 // transform (all variants)
 isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* pqr_regs_host,

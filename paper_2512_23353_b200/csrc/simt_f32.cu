@@ -201,15 +201,21 @@ __global__ void k_f32_combine(const float* __restrict__ G, int64_t N, int B, con
 
 }  // namespace
 
-isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq,
-                         cudaStream_t st) {
-  for (int base = 0; base <= B; base += kArgChunk) {
+isopo_status store_i64(const int64_t* host, int64_t n, int64_t* dev, cudaStream_t st) {
+  for (int64_t base = 0; base < n; base += kArgChunk) {
     OffsetArgs a;
-    const int n = std::min(kArgChunk, B + 1 - base);
-    for (int t = 0; t < n; ++t) a.v[t] = off_host[base + t];
-    k_store_offsets<<<1, kArgChunk, 0, st>>>(a, base, n, off_dev);
+    const int m = (int)std::min<int64_t>(kArgChunk, n - base);
+    for (int t = 0; t < m; ++t) a.v[t] = host[base + t];
+    k_store_offsets<<<1, kArgChunk, 0, st>>>(a, (int)base, m, dev);
     ISOPO_CUDA_TRY(cudaGetLastError());
   }
+  return ISOPO_OK;
+}
+
+isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq,
+                         cudaStream_t st) {
+  isopo_status s = store_i64(off_host, (int64_t)B + 1, off_dev, st);
+  if (s != ISOPO_OK) return s;
   const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
   {
     LaunchScope scope(kIdPrep, st);

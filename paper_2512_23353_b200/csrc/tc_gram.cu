@@ -34,19 +34,29 @@ constexpr uint32_t kTmemCols = 512;            // 2 buffers x (P 128 + Q 128) co
 
 struct GramParams {
   const int32_t* tokseq;
-  float* K;
+  float* K;       // Gram: K [B, B];  sampled: M^T [samples, B]
   int64_t T;
   int B, nT, d_in, d_out;
   int32_t* info;
+  int n_rows, n_row_tiles;  // sampled: sample rows and their 128-row tiles
 };
 
-// u = J (J + 1) / 2 + I with I <= J
-__device__ __forceinline__ void decode_pair(long long u, int& I, int& J) {
-  long long j = (long long)((sqrt(8.0 * (double)u + 1.0) - 1.0) * 0.5);
-  while ((j + 1) * (j + 2) / 2 <= u) ++j;
-  while (j * (j + 1) / 2 > u) --j;
-  J = (int)j;
-  I = (int)(u - j * (j + 1) / 2);
+// Work unit -> (row tile I, column tile J).  Gram: pairs I <= J of token tiles, u = J (J + 1) / 2 + I.
+// Sampled: every (sample tile, token tile).
+template <bool kSampled>
+__device__ __forceinline__ void decode_unit(const GramParams& p, long long u, int& I, int& J, bool& diag) {
+  if (kSampled) {
+    I = (int)(u % p.n_row_tiles);
+    J = (int)(u / p.n_row_tiles);
+    diag = false;
+  } else {
+    long long j = (long long)((sqrt(8.0 * (double)u + 1.0) - 1.0) * 0.5);
+    while ((j + 1) * (j + 2) / 2 <= u) ++j;
+    while (j * (j + 1) / 2 > u) --j;
+    J = (int)j;
+    I = (int)(u - j * (j + 1) / 2);
+    diag = I == J;
+  }
 }
 
 __device__ __forceinline__ float warp_sum_f(float v) {
@@ -66,8 +76,15 @@ __device__ __forceinline__ void flush_segment(float* __restrict__ K, int B, int 
   }
 }
 
+// kSampled = false: the Gram route, rows and columns are both token tiles (mapRX = mapX, mapRY = mapY).
+// kSampled = true: the token-sampled Fisher estimator of Algorithm 1: the rows are the sampled token
+// rows a0 = X[samples] (mapRX) and g0 = dY[samples] (mapRY), the columns all tokens, and
+//   M^T[j, i] = sum_{t in sequence i} (g0_j . dY_t)(a0_j . x_t) = g0_j . G_i a0_j      (Eq. one)
+// comes out of the same product-and-segment-sum epilogue without any symmetry weights.
+template <bool kSampled>
 __global__ void __launch_bounds__(kThreads, 1)
-k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY, GramParams p) {
+k_bf16_gram(const __grid_constant__ CUtensorMap mapRX, const __grid_constant__ CUtensorMap mapRY,
+            const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY, GramParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
@@ -93,28 +110,33 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  const long long total_units = (long long)p.nT * (p.nT + 1) / 2;
+  const long long total_units = kSampled ? (long long)p.n_row_tiles * p.nT : (long long)p.nT * (p.nT + 1) / 2;
   const int nkx = (p.d_in + kKF - 1) / kKF, nky = (p.d_out + kKF - 1) / kKF;
 
   if (warp == 0) {
     if (elect_one()) {
       prefetch_tensormap(&mapX);
       prefetch_tensormap(&mapY);
+      if (kSampled) {
+        prefetch_tensormap(&mapRX);
+        prefetch_tensormap(&mapRY);
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
         int I, J;
-        decode_pair(u, I, J);
-        const bool diag = I == J;
+        bool diag;
+        decode_unit<kSampled>(p, u, I, J, diag);
         for (int kb = 0; kb < nkx + nky; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdGram))) break;
-          const CUtensorMap* map = kb < nkx ? &mapX : &mapY;
+          const CUtensorMap* rmap = kb < nkx ? &mapRX : &mapRY;
+          const CUtensorMap* cmap = kb < nkx ? &mapX : &mapY;
           const int x = (kb < nkx ? kb : kb - nkx) * kKF;
           const uint32_t dst = smem_base + stage * kStageBytes;
           mbar_arrive_expect_tx(full_bar(stage), diag ? kOperandBytes : kStageBytes);
-          tma_load_2d(dst, map, x, I * kTT, full_bar(stage));
-          if (!diag) tma_load_2d(dst + kOperandBytes, map, x, J * kTT, full_bar(stage));
+          tma_load_2d(dst, rmap, x, I * kTT, full_bar(stage));
+          if (!diag) tma_load_2d(dst + kOperandBytes, cmap, x, J * kTT, full_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -127,8 +149,8 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
       bool ok = true;
       for (long long u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
         int I, J;
-        decode_pair(u, I, J);
-        const bool diag = I == J;
+        bool diag;
+        decode_unit<kSampled>(p, u, I, J, diag);
         if (!(ok = mbar_wait(accempty_bar(acc), acc_phase ^ 1u, abort_flag, p.info, kIdGram))) break;
         tc_fence_after_sync();
         for (int kb = 0; kb < nkx + nky; ++kb) {
@@ -159,12 +181,14 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
     uint32_t acc_phase = 0;
     for (long long u = blockIdx.x; u < total_units; u += gridDim.x) {
       int I, J;
-      decode_pair(u, I, J);
-      const bool diag = I == J;
+      bool diag;
+      decode_unit<kSampled>(p, u, I, J, diag);
       // sequence of this thread's row token and of every column token (clamped past the end; those
       // rows and columns are zero in P and Q)
+      // (sampled: the "row sequence" is the sample index, its results go to row `row_seq` of M^T;
+      // rows past the last sample are zero in P and Q and flush nothing)
       const int64_t trow = (int64_t)I * kTT + row;
-      const int row_seq = __ldg(p.tokseq + min(trow, p.T - 1));
+      const int row_seq = kSampled ? (int)trow : __ldg(p.tokseq + min(trow, p.T - 1));
       int csr[4];  // csr[g] of lane l = sequence of column token 32 g + l
 #pragma unroll
       for (int g = 0; g < 4; ++g) csr[g] = __ldg(p.tokseq + min((int64_t)J * kTT + g * 32 + lane, p.T - 1));
@@ -172,7 +196,7 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * 256;
       int cur = __shfl_sync(0xffffffffu, csr[0], 0);
-      float wseg = row_seq == cur ? 2.f : 1.f, run = 0.f;
+      float wseg = (!kSampled && row_seq == cur) ? 2.f : 1.f, run = 0.f;
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         const int c0 = g * 32;
@@ -194,7 +218,7 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
               flush_segment(p.K, p.B, row_seq, cur, run);
               run = 0.f;
               cur = sc;
-              wseg = row_seq == cur ? 2.f : 1.f;
+              wseg = (!kSampled && row_seq == cur) ? 2.f : 1.f;
             }
             const float h = __uint_as_float(pv[e]) * __uint_as_float(qv[e]);
             const float f = (!diag || c > row) ? wseg : (c == row ? 1.f : 0.f);
@@ -235,19 +259,44 @@ isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d
   int dev = 0, sms = 0;
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_gram, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_gram<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
-  GramParams p{tokseq, K, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info};
+  GramParams p{tokseq, K, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info, 0, 0};
   const long long units = (long long)p.nT * (p.nT + 1) / 2;
   const int grid = (int)std::min<long long>(units, sms);
   {
     LaunchScope scope(kIdGram, st);
-    k_bf16_gram<<<grid, kThreads, kSmemBytes, st>>>(mapX, mapY, p);
+    k_bf16_gram<false><<<grid, kThreads, kSmemBytes, st>>>(mapX, mapY, mapX, mapY, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   {
     LaunchScope scope(kIdMirror, st);
     k_mirror_upper_gram<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status bf16_sampled(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
+                          const void* A0, const void* G0, int n_samples, float* Mt, int32_t* info, cudaStream_t st) {
+  CUtensorMap mapX, mapY, mapRX, mapRY;
+  isopo_status s = make_map_2d_bf16(&mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kTT);
+  if (s != ISOPO_OK) return s;
+  if ((s = make_map_2d_bf16(&mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kTT)) != ISOPO_OK) return s;
+  // only the n_samples real rows are in bounds: the rest of the last 128-row tile reads as zero
+  if ((s = make_map_2d_bf16(&mapRX, A0, (uint64_t)n_samples, (uint64_t)d_in, (uint64_t)d_in, 64, kTT)) != ISOPO_OK) return s;
+  if ((s = make_map_2d_bf16(&mapRY, G0, (uint64_t)n_samples, (uint64_t)d_out, (uint64_t)d_out, 64, kTT)) != ISOPO_OK) return s;
+  int dev = 0, sms = 0;
+  ISOPO_CUDA_TRY(cudaGetDevice(&dev));
+  ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_gram<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  ISOPO_CUDA_TRY(cudaMemsetAsync(Mt, 0, sizeof(float) * (size_t)n_samples * B, st));
+  GramParams p{tokseq, Mt, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info, n_samples, (n_samples + kTT - 1) / kTT};
+  const long long units = (long long)p.n_row_tiles * p.nT;
+  const int grid = (int)std::min<long long>(units, sms);
+  {
+    LaunchScope scope(kIdSampled, st);
+    k_bf16_gram<true><<<grid, kThreads, kSmemBytes, st>>>(mapRX, mapRY, mapX, mapY, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
