@@ -237,12 +237,20 @@ def run_gpu(args):
     dt_code = b.BF16 if w.dtype == "bf16" else b.F32
     variant = b.VAR_INTERACTING if args.variant == "interacting" else b.VAR_NORMALISED
 
+    sampled = args.route == "sampled"
+    # Algorithm 1 draws its overlap samples with randperm: the bench draws them once, seeded, on the host
+    sample_rows = np.random.default_rng(w.seed + 17).permutation(T)[: args.samples].astype(np.int64)
     layers = []
     ws_bytes = 0
     for layer in w_layers:
         X, dY = wl.layer_inputs_device(w, layer, T, dev)
-        path = b.isopo_choose_path(dt_code, T, layer.d_in, layer.d_out, B)
-        ws_bytes = max(ws_bytes, b.isopo_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, path))
+        if sampled:
+            path = b.PATH_GRAM
+            ws_bytes = max(ws_bytes, b.isopo_sampled_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B,
+                                                                     len(sample_rows)))
+        else:
+            path = b.isopo_choose_path(dt_code, T, layer.d_in, layer.d_out, B)
+            ws_bytes = max(ws_bytes, b.isopo_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, path))
         layers.append({"layer": layer, "X": X, "dY": dY, "path": path,
                        "K": torch.empty((B, B), dtype=torch.float32, device=dev),
                        "c": torch.empty(B, dtype=torch.float32, device=dev),
@@ -254,18 +262,26 @@ def run_gpu(args):
     A = torch.from_numpy(A_host).to(dev)
     info = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    def step():
-        for L in layers:
+    def layer_calls(L):
+        if sampled:  # Algorithm 1: coefficients from sampled token rows, then the folded weight-gradient GEMM
+            b.isopo_sampled_coefficients(L["X"], L["dY"], off, sample_rows, A, L["lam"], L["c"], ws, info, L["F2"])
+        else:
             b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
             b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
-            b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+        b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+
+    def step():
+        for L in layers:
+            layer_calls(L)
 
     # the regulariser is an absolute number the caller carries from earlier minibatches:
-    # 1e-3 * mean(diag K), taken once from an untimed pass
+    # 1e-3 * mean(diag K) (stored route) or 1e-3 * mean(F^2) (sampled route), taken once from an untimed pass
+    for L in layers:
+        L["F2"] = torch.zeros(B, dtype=torch.float32, device=dev)
     step()
     torch.cuda.synchronize()
     for L in layers:
-        L["lam"] = 1e-3 * float(torch.diagonal(L["K"]).mean().item())
+        L["lam"] = 1e-3 * float((L["F2"] if sampled else torch.diagonal(L["K"])).mean().item())
     for _ in range(n_warm):
         step()
     torch.cuda.synchronize()
@@ -309,13 +325,23 @@ def run_gpu(args):
     flops_dw = sum(2.0 * T * L["layer"].d_in * L["layer"].d_out for L in layers)
     flops_k = sum(float(B) * B * L["layer"].d_in * L["layer"].d_out for L in layers)
     flops_comb = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers)
+    if sampled:
+        flops_k = sum(2.0 * T * len(sample_rows) * (L["layer"].d_in + L["layer"].d_out) for L in layers)
+        flops_comb = 0.0
     flops_step = flops_dw + flops_k + flops_comb
     step_tflops = flops_step / (ms_per_step * 1e-3) / 1e12
 
     # ---- roofline of the dominant kernel, from the events recorded inside the timed region ----
     dom = max(prof.items(), key=lambda kv: kv[1][0])[0] if prof else None
     roofline = None
-    if dom == "k_bf16_seq_grad":
+    if dom == "k_bf16_weight_grad":
+        ms_total, n = prof[dom]
+        achieved = flops_dw * args.steps / (ms_total * 1e-3) / 1e12
+        roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
+                    "avg_launch_ms": ms_total / n, "launches": n}
+    elif dom == "k_bf16_seq_grad":
         ms_total, n = prof[dom]
         achieved = flops_dw * args.steps / (ms_total * 1e-3) / 1e12
         # DRAM bytes per launch: the ncu capture of this kernel on a smaller case (gate_proj, 32 sequences:
@@ -344,9 +370,7 @@ def run_gpu(args):
     per_layer = []
     b.isopo_profile_enable(True)
     for L in layers:
-        b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
-        b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
-        b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+        layer_calls(L)
         pl = b.isopo_profile_collect()
         per_layer.append({"layer": L["layer"].name, **{k: round(v[0], 4) for k, v in pl.items()}})
     b.isopo_profile_enable(False)
@@ -386,9 +410,7 @@ def run_gpu(args):
             for L in layers:
                 L["X"].copy_(pinned[("X", L["layer"].d_in)], non_blocking=True)
                 L["dY"].copy_(pinned[("dY", L["layer"].d_out)], non_blocking=True)
-                b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
-                b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
-                b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+                layer_calls(L)
                 dW_host[id(L)].copy_(L["dW"], non_blocking=True)
 
         e2e_step()
@@ -416,11 +438,14 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-        "config": {"workload": args.workload, "B": B, "tokens": T, "variant": args.variant,
+        "config": {"workload": args.workload, "B": B, "tokens": T,
+                   "route": "sampled (Algorithm 1, %d token samples)" % len(sample_rows) if sampled else "stored gradients",
+                   "variant": "normalised (Algorithm 1)" if sampled else args.variant,
                    "layers": [f"{L['layer'].name}:{L['layer'].d_in}->{L['layer'].d_out}" for L in layers],
                    "paths": ["gram" if L["path"] == b.PATH_GRAM else "materialise" for L in layers],
                    "l2": "inputs larger than L2 (no flush needed)",
-                   "step": "layer_gram + transform_advantages + weight_grad for each projection"},
+                   "step": ("sampled_coefficients + weight_grad" if sampled else
+                            "layer_gram + transform_advantages + weight_grad") + " for each projection"},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(sum(v[1] for v in prof.values())),
@@ -446,6 +471,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llm_1p5b")
     ap.add_argument("--variant", default="interacting", choices=["interacting", "normalised"])
+    ap.add_argument("--route", default="stored", choices=["stored", "sampled"],
+                    help="stored: K from materialised per-sequence gradients (both variants); sampled: Algorithm 1's "
+                         "token-sampled Fisher norm + folded weight-gradient GEMM (non-interacting variant)")
+    ap.add_argument("--samples", type=int, default=128, help="n_overlap_samples of the sampled route")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--layers", default="", help="comma-separated projection names (default: all of the block)")

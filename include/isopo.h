@@ -229,7 +229,7 @@ ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, is
  * (host, ISOPO_NUM_KERNELS entries each, overwritten) and forgets them.  Launch counts are kept
  * even while event timing is disabled.  Not thread-safe; meant for benchmarks.
  */
-#define ISOPO_NUM_KERNELS 15
+#define ISOPO_NUM_KERNELS 16
 ISOPO_API void isopo_profile_enable(int on);
 ISOPO_API isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_kernel);
 ISOPO_API const char* isopo_kernel_name(int kernel_id);

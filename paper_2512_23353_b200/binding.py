@@ -31,7 +31,7 @@ EXPORTS = (
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
-NUM_KERNELS = 15
+NUM_KERNELS = 16
 
 
 class IsopoError(RuntimeError):

@@ -3,6 +3,7 @@
 // on the data and no CPU fallback.
 #include <cstdio>
 #include <cstring>
+#include <algorithm>
 #include <vector>
 
 #include "isopo_internal.h"
@@ -64,6 +65,9 @@ WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, iso
   p = align_up(p + sizeof(int32_t) * (size_t)T, 1024);
   L.off_kacc = p;
   if (dtype == ISOPO_F32) p = align_up(p + sizeof(double) * (size_t)B * (size_t)B, 1024);
+  L.off_scaled = p;
+  if (dtype == ISOPO_BF16 && resolved == ISOPO_PATH_GRAM)
+    p = align_up(p + (size_t)2 * (size_t)T * (size_t)std::min(d_in, d_out), 1024);
   L.off_G = p;
   if (dtype == ISOPO_BF16) {
     L.tiles_m = (d_out + kTileM - 1) / kTileM;
@@ -146,7 +150,7 @@ const char* isopo_kernel_name(int id) {
   static const char* names[kIdCount] = {"k_tokseq", "k_bf16_seq_grad", "k_bf16_ntk", "k_bf16_gram", "k_bf16_weight_grad",
                                         "k_bf16_combine", "k_transform", "k_mirror_upper", "k_f32_seq_grad",
                                         "k_f32_ntk", "k_f32_gram", "k_f32_weight_grad", "k_f32_combine",
-                                        "k_sampled", "k_sampled_aux"};
+                                        "k_sampled", "k_sampled_aux", "k_scale_rows"};
   return id >= 0 && id < kIdCount ? names[id] : "unknown";
 }
 
@@ -261,11 +265,17 @@ isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype,
   // GEMM over all tokens: refresh the token -> sequence map so the call also works on its own.
   int64_t* off_dev = (int64_t*)(w + L.off_offsets);
   int32_t* tokseq = (int32_t*)(w + L.off_tokseq);
-  s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
-  if (s != ISOPO_OK) return s;
-  if (dtype == ISOPO_F32)
+  if (dtype == ISOPO_F32) {
+    s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
+    if (s != ISOPO_OK) return s;
     return f32_weight_grad((const float*)X, (const float*)dY, T, d_in, d_out, coeffs, tokseq, dW, beta, st);
-  return bf16_weight_grad(X, dY, T, d_in, d_out, coeffs, tokseq, dW, beta, info, st);
+  }
+  // one scale per token, so that the kernel's scaler warps need a single independent load per row
+  float* tokscale = (float*)tokseq;
+  s = launch_tokscale(seq_offsets_host, B, T, off_dev, coeffs, tokscale, st);
+  if (s != ISOPO_OK) return s;
+  void* scaled = w + L.off_scaled;
+  return bf16_weight_grad(X, dY, T, d_in, d_out, tokscale, scaled, dW, beta, info, st);
 }
 
 }  // extern "C"

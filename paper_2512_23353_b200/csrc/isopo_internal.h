@@ -32,7 +32,8 @@ enum KernelId : int {
   kIdF32Combine = 12,
   kIdSampled = 13,     // M^T of the token-sampled estimator (tensor-core or float32 kernel)
   kIdSampledAux = 14,  // its gather and finishing kernels
-  kIdCount = 15
+  kIdScaleRows = 15,   // per-token scale of the narrower operand before the 2-CTA weight-gradient GEMM
+  kIdCount = 16
 };
 
 // Brackets one kernel launch with CUDA events while profiling is enabled (isopo_profile_enable);
@@ -60,8 +61,9 @@ class ProfilingPause {
 struct WsLayout {
   size_t off_offsets;  // int64 [B+1]
   size_t off_order;    // int32 [B]       (bf16 materialised path: sequences, longest first)
-  size_t off_tokseq;   // int32 [T]
+  size_t off_tokseq;   // int32 [T]: token -> sequence; the bf16 weight-gradient GEMM keeps float32 per-token scales here
   size_t off_kacc;     // float64 [B*B]   (float32 path: K accumulators)
+  size_t off_scaled;   // bf16 [T, min(d_in, d_out)]  (bf16 Gram path: the pre-scaled operand of the weight-gradient GEMM)
   size_t off_G;        // stored gradients (materialised path only)
   size_t total;
   int tiles_m, tiles_n;  // bf16 materialised layout: tiles per gradient
@@ -92,6 +94,9 @@ void set_cuda_error(cudaError_t e, const char* where);
 // ---- launchers (each enqueues on `st` and returns a status; none synchronises) ----
 
 isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq, cudaStream_t st);
+// offsets to the device and tokscale[t] = coeffs[sequence of token t] (float32 [T])
+isopo_status launch_tokscale(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, const float* coeffs,
+                             float* tokscale, cudaStream_t st);
 // n host values -> device array, passed as kernel arguments (no host-to-device copy)
 isopo_status store_i64(const int64_t* host, int64_t n, int64_t* dev, cudaStream_t st);
 // order_dev[k] = index of the k-th longest sequence (B <= 256)
@@ -119,8 +124,11 @@ isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out,
                           float beta, cudaStream_t st);
 isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
                        float* K, int32_t* info, cudaStream_t st);
-isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* coeffs,
-                              const int32_t* tokseq, float* dW, float beta, int32_t* info, cudaStream_t st);
+isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* tokscale,
+                              void* scaled, float* dW, float beta, int32_t* info, cudaStream_t st);
+
+isopo_status bf16_weight_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* tokscale,
+                                   void* scaled, float* dW, float beta, int32_t* info, cudaStream_t st);
 
 // token-sampled estimator of Algorithm 1
 isopo_status bf16_sampled(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,

@@ -37,6 +37,19 @@ __global__ void k_tokseq(const int64_t* __restrict__ off, int B, int64_t T, int3
   }
 }
 
+// tokscale[t] = coeffs[sequence of token t]: what the folded weight-gradient GEMM multiplies row t by.
+__global__ void k_tokscale(const int64_t* __restrict__ off, int B, int64_t T, const float* __restrict__ coeffs,
+                           float* __restrict__ tokscale) {
+  for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
+    int lo = 0, hi = B;  // invariant: off[lo] <= t < off[hi]
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (off[mid] <= t) lo = mid; else hi = mid;
+    }
+    tokscale[t] = coeffs[lo];
+  }
+}
+
 // Accumulates, for tokens [t0, t1), acc[4][4] += w_t * dY[t, m0+4ty+a] * X[t, n0+4tx+b].
 template <bool kScaled>
 __device__ __forceinline__ void gemm_tokens(const float* __restrict__ X, const float* __restrict__ dY, int d_in,
@@ -220,6 +233,19 @@ isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off
   {
     LaunchScope scope(kIdPrep, st);
     k_tokseq<<<grid, 256, 0, st>>>(off_dev, B, T, tokseq);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status launch_tokscale(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, const float* coeffs,
+                             float* tokscale, cudaStream_t st) {
+  isopo_status s = store_i64(off_host, (int64_t)B + 1, off_dev, st);
+  if (s != ISOPO_OK) return s;
+  const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
+  {
+    LaunchScope scope(kIdPrep, st);
+    k_tokscale<<<grid, 256, 0, st>>>(off_dev, B, T, coeffs, tokscale);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

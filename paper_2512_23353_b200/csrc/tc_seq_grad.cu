@@ -49,8 +49,7 @@ struct SeqGradParams {
   int B, tiles_m, tiles_n;
   int32_t* info;
   // folded weight-gradient GEMM only
-  const float* coeffs;
-  const int32_t* tokseq;
+  const float* tokscale;  // coefficient of every token's sequence
   float* dW;
   int64_t T, slab;  // tokens per work unit (a multiple of 64)
   int nslabs, d_in, d_out;
@@ -285,7 +284,7 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
       const int nkb = (int)((t1 - t0 + kKB - 1) / kKB);
       for (int kb = 0; kb < nkb; ++kb) {
         const int64_t t = t0 + (int64_t)kb * kKB + r;
-        const float c = t < t1 ? __ldg(p.coeffs + __ldg(p.tokseq + t)) : 0.f;
+        const float c = t < t1 ? __ldg(p.tokscale + t) : 0.f;
         if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.info, kIdSeqGrad))) break;
         const uint32_t a_addr = smem_base + stage * kStageBytes + r * 128 + h * 64;
 #pragma unroll
@@ -360,8 +359,12 @@ isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, i
   return ISOPO_OK;
 }
 
-isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* coeffs,
-                              const int32_t* tokseq, float* dW, float beta, int32_t* info, cudaStream_t st) {
+isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* tokscale,
+                              void* scaled, float* dW, float beta, int32_t* info, cudaStream_t st) {
+  {  // 2-CTA tiles when they waste little (see bf16_seq_grad)
+    const int tiles_m = (d_out + kTileM - 1) / kTileM;
+    if (tiles_m % 2 == 0 || tiles_m >= 7) return bf16_weight_grad_pair(X, dY, T, d_in, d_out, tokscale, scaled, dW, beta, info, st);
+  }
   CUtensorMap mapY, mapX;
   isopo_status s = make_maps(&mapY, &mapX, X, dY, T, d_in, d_out);
   if (s != ISOPO_OK) return s;
@@ -372,7 +375,7 @@ isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in
   SeqGradParams p{};
   p.tiles_m = (d_out + kTileM - 1) / kTileM;
   p.tiles_n = (d_in + kTileN - 1) / kTileN;
-  p.info = info; p.coeffs = coeffs; p.tokseq = tokseq; p.dW = dW; p.T = T; p.d_in = d_in; p.d_out = d_out;
+  p.info = info; p.tokscale = tokscale; p.dW = dW; p.T = T; p.d_in = d_in; p.d_out = d_out;
   // token slabs: enough (tile, slab) units to fill the machine about twice, each slab a multiple of 64 tokens
   const long long tiles = (long long)p.tiles_m * p.tiles_n;
   const long long kblocks = (T + kKB - 1) / kKB;
