@@ -261,7 +261,8 @@ isopo_status bf16_weight_grad_pair(const void* X, const void* dY, int64_t T, int
   p.ptiles_m = ((d_out + kHalf - 1) / kHalf + 1) / 2;
   p.tiles_n = (d_in + kPairN - 1) / kPairN;
   // token slabs: about eight (tile, slab) units per pair so that the round-robin share is even; every
-  // slab a multiple of the stage depth
+  // slab a multiple of the stage depth.  (Slabs small enough for their rows to stay in L2 across the
+  // waves of tiles were measured slower: the float32 reductions into dW grow with the slab count.)
   const long long ptiles = (long long)p.ptiles_m * p.tiles_n, pairs = resident_pairs[dev];
   const long long kblocks = (T + kKB - 1) / kKB;
   long long nslabs = std::max<long long>(1, std::min<long long>(kblocks, (8 * pairs + ptiles - 1) / ptiles));
