@@ -95,8 +95,9 @@ ISOPO_API isopo_path isopo_choose_path(isopo_dtype dtype, int64_t T, int d_in, i
  * Bytes of device workspace the three calls of one layer need for `path` (AUTO allowed).
  * The workspace holds the device copy of the offsets, the token -> sequence map and, on the
  * materialised path, all B per-sequence gradients (bf16 for ISOPO_BF16, float32 for ISOPO_F32)
- * in a tile-blocked order private to the library.  It must be 1024-byte aligned.  Returns 0 for
- * invalid sizes.
+ * in a piece-blocked order private to the library; on the bf16 Gram path, the per-token-scaled
+ * copy of the narrower of X and dY that isopo_weight_grad feeds to its GEMM
+ * (2 * T * min(d_in, d_out) bytes).  It must be 1024-byte aligned.  Returns 0 for invalid sizes.
  */
 ISOPO_API size_t isopo_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path path);
 
@@ -147,7 +148,9 @@ ISOPO_API isopo_status isopo_transform_advantages(const float* K, const float* A
  *
  * `path` must be the value given to isopo_layer_gram for this layer (AUTO resolves identically).
  * MATERIALISE: streams the G_i left in the workspace by isopo_layer_gram.  GRAM: one GEMM over all
- * tokens, dW = (coeffs[seq(t)] * dY)^T X, with the per-token scale folded into the operand.
+ * tokens, dW = (coeffs[seq(t)] * dY)^T X, with the per-token scale applied to the narrower operand
+ * (rounded to nearest even in bf16) in one pass before the GEMM, or, for small layers, to the rows
+ * as they land in shared memory.
  *
  *   coeffs  dev, float32 [B]
  *   dW      dev, float32 [d_out, d_in] row-major (the layout of `grad_out.T @ act_in`)
