@@ -143,6 +143,32 @@ ISOPO_API isopo_status isopo_transform_advantages(const float* K, const float* A
                                         const float* opt_pqr_regs, float* coeffs, int32_t* info, void* cuda_stream);
 
 /*
+ * Relative regularisation (Alg. 1: "use e.g. EMA of trailing minibatch means for the regularization";
+ * generalised re-scaling figure: reg(val) = val + regularization * expectation(val); Sec. 4:
+ * "regularization factor 1.0 * E[mean(D)] ... EMA over minibatches with 0.9 decay").
+ *
+ * isopo_reg_ema_update folds one microbatch's K into running means kept on the device, so that the
+ * whole layer (gram -> update -> transform -> weight_grad) runs without the host reading anything:
+ *     state[0] = E[F_i^2]   state[1] = E[K_ii] = E[mean(D)], the mean eigenvalue of K
+ *     state[2] = E[F_i^2 / K_ii]   state[3] = number of updates so far
+ * with F_i^2 = sum_j K_ij^2 / sum_j K_jj.  The caller zeroes the four floats once; the first update
+ * stores the microbatch means, later ones blend  s <- decay * s + (1 - decay) * mean,  0 <= decay < 1.
+ *
+ * isopo_transform_advantages_rel is isopo_transform_advantages with the regulariser given as a
+ * factor of the matching running mean, read on the device (the state as updated so far, i.e.
+ * including the current microbatch if the update was issued first):
+ *     NORMALISED(_RAW): lambda = factor * E[F^2]      DIRECTION: lambda = factor * E[F^2 / K_ii]
+ *     EUCLID, INTERACTING: lambda = factor * E[K_ii]
+ *     GENERAL: opt_pqr_factors = {p, q, r, factor_F, factor_G, factor_rel} (host), `factor` ignored.
+ *
+ *   state   dev, float32 [4]
+ */
+ISOPO_API isopo_status isopo_reg_ema_update(const float* K, int B, float decay, float* state, void* cuda_stream);
+ISOPO_API isopo_status isopo_transform_advantages_rel(const float* K, const float* A, int B, isopo_variant variant,
+                                                      float factor, const float* opt_pqr_factors, const float* state,
+                                                      float* coeffs, int32_t* info, void* cuda_stream);
+
+/*
  * isopo_weight_grad: dW = beta * dW + sum_i coeffs[i] * G_i   (Alg. 1 "grad += advantages * rescaled
  * gradient" and "mod.grad += grad"; Alg. 2 "stack(seq_grads) @ advantages_preconditioned").
  *

@@ -174,6 +174,27 @@ def transform_advantages(K, A, variant, lam=0.0, pqr=None, regs=None):
     raise ValueError(f"unknown variant {variant!r}")
 
 
+def regulariser_means(K):
+    """Microbatch means of the quantities the relative regulariser is added to (generalised
+    re-scaling figure: `reg(val) = val + regularization * expectation(val)`):
+    (mean_i F_i^2, mean_i ||G_i||^2, mean_i F_i^2/||G_i||^2).  mean_i ||G_i||^2 = tr K / B is also the
+    mean eigenvalue `mean(D)` that the interacting experiment regularises with."""
+    K = _f64(K)
+    F2 = fisher_norm_sq(K)
+    n2 = np.diag(K)
+    return np.array([np.mean(F2), np.mean(n2), np.mean(F2 / n2)])
+
+
+def ema_update(state, means, decay):
+    """Running mean over microbatches ("EMA over minibatches with 0.9 decay").  state = (values[3],
+    number of updates); the first update takes the means themselves."""
+    values, n = state
+    means = _f64(means)
+    if n == 0:
+        return means.copy(), 1
+    return decay * _f64(values) + (1.0 - decay) * means, n + 1
+
+
 def weight_gradient(G, c):
     """dW = sum_i c_i G_i (Algorithm 1: `grad += advantages[seq_id] * rescaled
     seq_logprob_grad`; Algorithm 2: `stack(seq_grads, -1) @ advantages_preconditioned`)."""

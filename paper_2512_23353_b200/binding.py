@@ -28,6 +28,7 @@ EXPORTS = (
     "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad",
     "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
     "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
+    "isopo_reg_ema_update", "isopo_transform_advantages_rel",
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
@@ -74,6 +75,11 @@ def _load():
     lib.isopo_sampled_coefficients.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
                                                c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_float, c.c_void_p,
                                                c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.isopo_reg_ema_update.restype = c.c_int
+    lib.isopo_reg_ema_update.argtypes = [c.c_void_p, c.c_int, c.c_float, c.c_void_p, c.c_void_p]
+    lib.isopo_transform_advantages_rel.restype = c.c_int
+    lib.isopo_transform_advantages_rel.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
+                                                   c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.isopo_profile_enable.restype = None
     lib.isopo_profile_enable.argtypes = [c.c_int]
     lib.isopo_profile_collect.restype = c.c_int
@@ -173,6 +179,30 @@ def isopo_transform_advantages(K: torch.Tensor, A: torch.Tensor, variant: int, l
                                         g.ctypes.data if g is not None else None, coeffs.data_ptr(),
                                         info.data_ptr(), _stream())
     _check(st, "isopo_transform_advantages")
+
+
+def isopo_reg_ema_update(K: torch.Tensor, decay: float, state: torch.Tensor) -> None:
+    """Folds this microbatch's K into the running means `state` (device float32 [4], zeroed once by the caller)."""
+    B = K.shape[0]
+    assert K.dtype == torch.float32 and K.is_contiguous() and K.numel() == B * B
+    assert state.dtype == torch.float32 and state.numel() == 4 and state.is_cuda
+    _check(lib.isopo_reg_ema_update(K.data_ptr(), B, float(decay), state.data_ptr(), _stream()), "isopo_reg_ema_update")
+
+
+def isopo_transform_advantages_rel(K: torch.Tensor, A: torch.Tensor, variant: int, factor: float, state: torch.Tensor,
+                                   coeffs: torch.Tensor, info: torch.Tensor, pqr_factors=None) -> None:
+    """isopo_transform_advantages with the regulariser = factor x the running mean kept in `state`."""
+    B = A.numel()
+    assert K.dtype == torch.float32 and A.dtype == torch.float32 and coeffs.dtype == torch.float32
+    assert K.is_contiguous() and K.numel() == B * B and coeffs.numel() == B and state.numel() == 4
+    g = None
+    if pqr_factors is not None:
+        g = np.ascontiguousarray(np.asarray(pqr_factors, dtype=np.float32))
+        assert g.shape == (6,)
+    st = lib.isopo_transform_advantages_rel(K.data_ptr(), A.data_ptr(), B, variant, float(factor),
+                                            g.ctypes.data if g is not None else None, state.data_ptr(),
+                                            coeffs.data_ptr(), info.data_ptr(), _stream())
+    _check(st, "isopo_transform_advantages_rel")
 
 
 def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, seq_offsets, dW: torch.Tensor,

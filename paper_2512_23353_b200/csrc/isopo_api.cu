@@ -242,7 +242,23 @@ isopo_status isopo_transform_advantages(const float* K, const float* A, int B, i
   if (!(lambda >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
   if (variant == ISOPO_VAR_GENERAL && !opt_pqr_regs) return ISOPO_ERR_INVALID_ARG;
   if (variant == ISOPO_VAR_INTERACTING && B > 256) return ISOPO_ERR_UNSUPPORTED;
-  return transform(K, A, B, variant, lambda, opt_pqr_regs, coeffs, info, (cudaStream_t)cuda_stream);
+  return transform(K, A, B, variant, lambda, opt_pqr_regs, nullptr, coeffs, info, (cudaStream_t)cuda_stream);
+}
+
+isopo_status isopo_reg_ema_update(const float* K, int B, float decay, float* state, void* cuda_stream) {
+  if (!K || !state || B < 1 || !(decay >= 0.0f && decay < 1.0f)) return ISOPO_ERR_INVALID_ARG;
+  return reg_ema_update(K, B, decay, state, (cudaStream_t)cuda_stream);
+}
+
+isopo_status isopo_transform_advantages_rel(const float* K, const float* A, int B, isopo_variant variant, float factor,
+                                            const float* opt_pqr_factors, const float* state, float* coeffs,
+                                            int32_t* info, void* cuda_stream) {
+  if (!K || !A || !coeffs || !info || !state || B < 1) return ISOPO_ERR_INVALID_ARG;
+  if ((int)variant < 0 || (int)variant > (int)ISOPO_VAR_NORMALISED_RAW) return ISOPO_ERR_INVALID_ARG;
+  if (!(factor >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
+  if (variant == ISOPO_VAR_GENERAL && !opt_pqr_factors) return ISOPO_ERR_INVALID_ARG;
+  if (variant == ISOPO_VAR_INTERACTING && B > 256) return ISOPO_ERR_UNSUPPORTED;
+  return transform(K, A, B, variant, factor, opt_pqr_factors, state, coeffs, info, (cudaStream_t)cuda_stream);
 }
 
 isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,

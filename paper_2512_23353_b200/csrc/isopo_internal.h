@@ -140,6 +140,7 @@ isopo_status sampled_coefficients(const void* X, const void* dY, isopo_dtype dty
 
 // transform (all variants)
 isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* pqr_regs_host,
-                       float* coeffs, int32_t* info, cudaStream_t st);
+                       const float* rel_state, float* coeffs, int32_t* info, cudaStream_t st);
+isopo_status reg_ema_update(const float* K, int B, float decay, float* state, cudaStream_t st);
 
 }  // namespace isopo

@@ -22,6 +22,8 @@ struct TransformParams {
   int variant;
   float lambda;
   float p, q, r, reg_F, reg_G, reg_rel;
+  const float* rel_state;  // NULL, or the running means {E[F^2], E[||G||^2], E[F^2/||G||^2], updates}: the
+                           // regularisers above are then factors of these (relative regularisation)
 };
 
 
@@ -211,6 +213,19 @@ __global__ void __launch_bounds__(kThreads) k_transform(TransformParams P) {
   __shared__ int s_fail;
   const int B = P.B, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kThreads / 32;
   const float* __restrict__ K = P.K;
+  if (P.rel_state) {
+    // reg(val) = val + regularization * expectation(val) of the generalised re-scaling figure: each
+    // regulariser is its factor times the running mean of the quantity it is added to
+    const float eF = P.rel_state[0], eG = P.rel_state[1], eR = P.rel_state[2];
+    switch (P.variant) {
+      case ISOPO_VAR_NORMALISED:
+      case ISOPO_VAR_NORMALISED_RAW: P.lambda *= eF; break;
+      case ISOPO_VAR_DIRECTION: P.lambda *= eR; break;
+      case ISOPO_VAR_EUCLID:
+      case ISOPO_VAR_INTERACTING: P.lambda *= eG; break;  // mean eigenvalue of K = tr K / B = E[||G||^2]
+      default: P.reg_F *= eF; P.reg_G *= eG; P.reg_rel *= eR;
+    }
+  }
 
   if (P.variant == ISOPO_VAR_REINFORCE) {
     for (int i = tid; i < B; i += kThreads) P.coeffs[i] = P.A[i];
@@ -410,12 +425,59 @@ __global__ void __launch_bounds__(kThreads) k_transform(TransformParams P) {
   for (int i = tid; i < B; i += kThreads) P.coeffs[i] = (float)sol[i];
 }
 
+// Running means for the relative regulariser.  state = {E[F^2], E[||G||^2], E[F^2 / ||G||^2], number of updates};
+// the first update stores this microbatch's means, later ones blend: s <- decay * s + (1 - decay) * mean.
+__global__ void __launch_bounds__(kThreads) k_reg_ema(const float* __restrict__ K, int B, float decay,
+                                                      float* __restrict__ state) {
+  __shared__ double s_trace, s_f2, s_rel;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kThreads / 32;
+  double tr = 0.0;
+  for (int i = tid; i < B; i += kThreads) tr += (double)K[(size_t)i * B + i];
+  tr = warp_sum(tr);
+  if (tid == 0) { s_trace = 0.0; s_f2 = 0.0; s_rel = 0.0; }
+  __syncthreads();
+  if (lane == 0) atomicAdd(&s_trace, tr);
+  __syncthreads();
+  const double trace = s_trace;
+  double f2_sum = 0.0, rel_sum = 0.0;
+  for (int i = warp; i < B; i += nwarps) {
+    double sq = 0.0;
+    for (int j = lane; j < B; j += 32) {
+      const double kij = (double)K[(size_t)i * B + j];
+      sq += kij * kij;
+    }
+    sq = warp_sum(sq);
+    const double F2 = sq / trace;
+    f2_sum += F2;
+    rel_sum += F2 / (double)K[(size_t)i * B + i];
+  }
+  if (lane == 0) { atomicAdd(&s_f2, f2_sum); atomicAdd(&s_rel, rel_sum); }
+  __syncthreads();
+  if (tid == 0) {
+    const double m[3] = {s_f2 / B, trace / B, s_rel / B};
+    const bool first = state[3] == 0.f;
+    for (int k = 0; k < 3; ++k)
+      state[k] = (float)(first ? m[k] : (double)decay * (double)state[k] + (1.0 - (double)decay) * m[k]);
+    state[3] += 1.f;
+  }
+}
+
 }  // namespace
 
+isopo_status reg_ema_update(const float* K, int B, float decay, float* state, cudaStream_t st) {
+  {
+    LaunchScope scope(kIdTransform, st);
+    k_reg_ema<<<1, kThreads, 0, st>>>(K, B, decay, state);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
 isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* g,
-                       float* coeffs, int32_t* info, cudaStream_t st) {
+                       const float* rel_state, float* coeffs, int32_t* info, cudaStream_t st) {
   TransformParams P{};
   P.K = K; P.A = A; P.coeffs = coeffs; P.info = info; P.B = B; P.variant = (int)v; P.lambda = lambda;
+  P.rel_state = rel_state;
   if (v == ISOPO_VAR_GENERAL) { P.p = g[0]; P.q = g[1]; P.r = g[2]; P.reg_F = g[3]; P.reg_G = g[4]; P.reg_rel = g[5]; }
   size_t smem = 0;
   if (v == ISOPO_VAR_INTERACTING) {

@@ -375,6 +375,29 @@ def test_sampled_estimator_invariances_and_bound():
     np.testing.assert_allclose(dW, sum(A[i] / np.sqrt(F2[i] + 0.3) * G[i] for i in range(6)), rtol=1e-11)
 
 
+# ----------------------------------------------------------------------------- relative regulariser
+def test_regulariser_means_and_ema():
+    X, dY, off, _ = _problem(91, B=7)
+    K = orc.ntk(orc.sequence_gradients(X, dY, off))
+    m = orc.regulariser_means(K)
+    # mean ||G_i||^2 is the mean eigenvalue of K, the statistic the interacting experiment names
+    np.testing.assert_allclose(m[1], np.mean(np.linalg.eigvalsh(K)), rtol=1e-12)
+    # diagonal K: F_i^2 = K_ii^2 / tr K, F_i^2 / K_ii = K_ii / tr K, whose mean is exactly 1 / B
+    Kd = np.diag([1.0, 2.0, 5.0])
+    np.testing.assert_allclose(orc.regulariser_means(Kd), [30.0 / 8.0 / 3.0, 8.0 / 3.0, 1.0 / 3.0], rtol=1e-14)
+    # EMA: first update takes the value; n equal updates stay there; the closed form of the geometric weights
+    s = (np.zeros(3), 0)
+    s = orc.ema_update(s, [4.0, 4.0, 4.0], 0.9)
+    np.testing.assert_allclose(s[0], 4.0)
+    for _ in range(5):
+        s = orc.ema_update(s, [4.0, 4.0, 4.0], 0.9)
+    np.testing.assert_allclose(s[0], 4.0, rtol=1e-14)
+    s = orc.ema_update(s, [14.0, 4.0, 4.0], 0.9)
+    s = orc.ema_update(s, [4.0, 4.0, 4.0], 0.9)
+    np.testing.assert_allclose(s[0][0], 4.0 + 0.9 * 0.1 * 10.0, rtol=1e-14)
+    assert s[1] == 8
+
+
 def test_pins_catch_planted_mistakes(monkeypatch):
     """Each mistake planted in the oracle (an off-by-one partition, a one-sided kernel fill, a
     dropped normalisation, a wrong regulariser sign) makes a pin above fail."""

@@ -72,3 +72,36 @@ def test_not_pd_pivot_index_in_a_later_block(b):
     b.isopo_transform_advantages(Kd, torch.ones(B, device="cuda"), b.VAR_INTERACTING, 0.0, c, info)
     torch.cuda.synchronize()
     assert int(info.item()) == 41
+
+
+def test_relative_regulariser_runs_without_host_values(b):
+    """gram -> isopo_reg_ema_update -> isopo_transform_advantages_rel over three microbatches: the
+    running means and the coefficients must equal the oracle's, which is handed the same K matrices."""
+    rng = np.random.default_rng(3)
+    B = 48
+    state = torch.zeros(4, device="cuda")
+    o_state = (np.zeros(3), 0)
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step in range(3):
+        M = rng.standard_normal((B, 300)) * (1.0 + step)
+        K64 = M @ M.T
+        K = torch.from_numpy(K64.astype(np.float32)).cuda()
+        A = torch.from_numpy(rng.standard_normal(B).astype(np.float32)).cuda()
+        K64 = K.double().cpu().numpy()
+        b.isopo_reg_ema_update(K, 0.9, state)
+        o_state = orc.ema_update(o_state, orc.regulariser_means(K64), 0.9)
+        np.testing.assert_allclose(state[:3].cpu().numpy(), o_state[0], rtol=2e-6)
+        assert int(state[3].item()) == step + 1
+        for variant, name, idx in ((b.VAR_NORMALISED, orc.NORMALISED, 0), (b.VAR_DIRECTION, orc.DIRECTION, 2),
+                                   (b.VAR_EUCLID, orc.EUCLID, 1), (b.VAR_INTERACTING, orc.INTERACTING, 1)):
+            c = torch.empty(B, device="cuda")
+            b.isopo_transform_advantages_rel(K, A, variant, 0.5, state, c, info)
+            want = orc.transform_advantages(K64, A.double().cpu().numpy(), name, 0.5 * o_state[0][idx])
+            assert rel_fro(c.cpu().numpy(), want) <= 1e-5, (step, name)
+        g = [-1.0, -0.5, 0.25, 0.5, 2.0, 0.1]
+        c = torch.empty(B, device="cuda")
+        b.isopo_transform_advantages_rel(K, A, b.VAR_GENERAL, 0.0, state, c, info, g)
+        want = orc.transform_advantages(K64, A.double().cpu().numpy(), orc.GENERAL, 0.0, tuple(g[:3]),
+                                        (g[3] * o_state[0][0], g[4] * o_state[0][1], g[5] * o_state[0][2]))
+        assert rel_fro(c.cpu().numpy(), want) <= 1e-5
+    assert int(info.item()) == 0
