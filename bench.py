@@ -325,6 +325,11 @@ def run_gpu(args):
     flops_dw = sum(2.0 * T * L["layer"].d_in * L["layer"].d_out for L in layers)
     flops_k = sum(float(B) * B * L["layer"].d_in * L["layer"].d_out for L in layers)
     flops_comb = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers)
+    if not sampled:  # layers on the Gram route: token Grams instead of the K pass and the combine
+        gram_layers = [L for L in layers if L["path"] == b.PATH_GRAM]
+        flops_k = sum(float(B) * B * L["layer"].d_in * L["layer"].d_out for L in layers if L["path"] != b.PATH_GRAM) + \
+            sum(float(L["layer"].d_in + L["layer"].d_out) * T * T for L in gram_layers)
+        flops_comb = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers if L["path"] != b.PATH_GRAM)
     if sampled:
         flops_k = sum(2.0 * T * len(sample_rows) * (L["layer"].d_in + L["layer"].d_out) for L in layers)
         flops_comb = 0.0
@@ -340,6 +345,15 @@ def run_gpu(args):
         roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
                     "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
+                    "avg_launch_ms": ms_total / n, "launches": n}
+    elif dom == "k_bf16_gram":
+        # Gram route: (d_in + d_out) T^2 flop per layer (symmetric half of the two token Grams)
+        ms_total, n = prof[dom]
+        flops_gram = sum(float(L["layer"].d_in + L["layer"].d_out) * T * T for L in layers if L["path"] == b.PATH_GRAM)
+        achieved = flops_gram * args.steps / (ms_total * 1e-3) / 1e12
+        roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                    "peak_source": f"{peaks['source']} burst bf16 (short kernels; sustained {peaks['bf16_tflops_sustained']})",
                     "avg_launch_ms": ms_total / n, "launches": n}
     elif dom == "k_bf16_seq_grad":
         ms_total, n = prof[dom]

@@ -59,6 +59,9 @@ WORKLOADS = {
     # small-LLM block: d_model 896, FFN 4864 (kv width 128 assumed), 64 sequences of 128..1024 tokens
     "small_llm": Workload("small_llm", "bf16", 64, "uniform", 128, 1024, 8, "uniform",
                           _block(896, 4864, 128), seed=1002),
+    # short rollouts on the small-LLM block (256 sequences of 16..64 tokens): the regime where the Gram route is cheaper
+    "short_rollouts": Workload("short_rollouts", "bf16", 256, "uniform", 16, 64, 8, "uniform",
+                               _block(896, 4864, 128), seed=1006),
     # 1.5B-class block: d_model 1536, FFN 8960, GQA kv width 256, 32 prompts x 8 samples
     "llm_1p5b": Workload("llm_1p5b", "bf16", 256, "loguniform", 256, 4096, 8, "uniform",
                          _block(1536, 8960, 256), seed=1003),
