@@ -90,7 +90,7 @@ def test_wide_projection_sampled(b, workload, name, n_sample):
     K_gpu = K.cpu().numpy()[np.ix_(pick, pick)]
     assert rel_fro(K_gpu, K_s) <= TOL
     assert np.max(np.abs(np.diag(K_gpu) - np.diag(K_s)) / np.diag(K_s)) <= TOL
-    # off-diagonal entries are tiny for independent tokens: judge them on the Cauchy-Schwarz scale sqrt(K_ii K_jj)
+    # off-diagonal entries are tiny for independent tokens: measure them on the Cauchy-Schwarz scale sqrt(K_ii K_jj)
     assert np.max(np.abs(K_gpu - K_s) / np.sqrt(np.outer(np.diag(K_s), np.diag(K_s)))) <= TOL
     del G_s
     # a sampled block of dW over all sequences, with the GPU's own coefficients
