@@ -15,7 +15,9 @@
 //   warp 0      TMA producer: [128 tokens] x [64 features] boxes of X then of dY, 6-stage ring
 //   warp 1      MMA issuer: tcgen05.mma 128 x 128 x 16, K-major operands
 //   warps 2-5   epilogue: tcgen05.ld of P and Q, product, segmented sums, float atomics into K
+
 #include "tc_common.cuh"
+#include "tc_gram_epilogue.cuh"
 
 namespace isopo {
 
@@ -39,9 +41,10 @@ struct GramParams {
   int B, nT, d_in, d_out;
   int32_t* info;
   int n_rows, n_row_tiles;  // sampled: sample rows and their 128-row tiles
+  int strip;                // Gram: tile columns per strip of the pair order
 };
 
-// Work unit -> (row tile I, column tile J).  Gram: pairs I <= J of token tiles, u = J (J + 1) / 2 + I.
+// Work unit -> (row tile I, column tile J).  Gram: pairs I <= J of token tiles in strip order.
 // Sampled: every (sample tile, token tile).
 template <bool kSampled>
 __device__ __forceinline__ void decode_unit(const GramParams& p, long long u, int& I, int& J, bool& diag) {
@@ -50,29 +53,8 @@ __device__ __forceinline__ void decode_unit(const GramParams& p, long long u, in
     J = (int)(u / p.n_row_tiles);
     diag = false;
   } else {
-    long long j = (long long)((sqrt(8.0 * (double)u + 1.0) - 1.0) * 0.5);
-    while ((j + 1) * (j + 2) / 2 <= u) ++j;
-    while (j * (j + 1) / 2 > u) --j;
-    J = (int)j;
-    I = (int)(u - j * (j + 1) / 2);
+    decode_pair_strips(u, p.nT, p.strip, I, J);
     diag = I == J;
-  }
-}
-
-__device__ __forceinline__ float warp_sum_f(float v) {
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// Adds `v` (one value per lane, lane = tile row) into K[row_seq][col_seq]; one atomic per warp when
-// all rows of the warp belong to the same sequence.
-__device__ __forceinline__ void flush_segment(float* __restrict__ K, int B, int row_seq, int col_seq, float v) {
-  const unsigned same = __match_any_sync(0xffffffffu, row_seq);
-  if (same == 0xffffffffu) {
-    v = warp_sum_f(v);
-    if ((threadIdx.x & 31) == 0 && v != 0.f) atomicAdd(&K[(size_t)row_seq * B + col_seq], v);
-  } else if (v != 0.f) {
-    atomicAdd(&K[(size_t)row_seq * B + col_seq], v);
   }
 }
 
@@ -189,44 +171,25 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapRX, const __grid_constant__ C
       // rows past the last sample are zero in P and Q and flush nothing)
       const int64_t trow = (int64_t)I * kTT + row;
       const int row_seq = kSampled ? (int)trow : __ldg(p.tokseq + min(trow, p.T - 1));
-      int csr[4];  // csr[g] of lane l = sequence of column token 32 g + l
-#pragma unroll
-      for (int g = 0; g < 4; ++g) csr[g] = __ldg(p.tokseq + min((int64_t)J * kTT + g * 32 + lane, p.T - 1));
+      auto col_seq = [&](int g) { return __ldg(p.tokseq + min((int64_t)J * kTT + g * 32 + lane, p.T - 1)); };
+      int cs = col_seq(0);  // sequence of column token 32 g + lane
       if (!mbar_wait(accfull_bar(acc), acc_phase, abort_flag, p.info, kIdGram)) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * 256;
-      int cur = __shfl_sync(0xffffffffu, csr[0], 0);
+      const RowSegments rows = row_segments(row_seq);
+      int cur = __shfl_sync(0xffffffffu, cs, 0);
       float wseg = (!kSampled && row_seq == cur) ? 2.f : 1.f, run = 0.f;
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        const int c0 = g * 32;
+#pragma unroll 1
+      for (int g = 0; g < kTT / 32; ++g) {
+        const int cs_next = g + 1 < kTT / 32 ? col_seq(g + 1) : 0;
         uint32_t pv[32], qv[32];
-        tmem_ld32(taddr + c0, pv);
-        tmem_ld32(taddr + 128 + c0, qv);
+        tmem_ld32(taddr + g * 32, pv);
+        tmem_ld32(taddr + 128 + g * 32, qv);
         tmem_ld_wait();
-        const bool one_segment = __shfl_sync(0xffffffffu, csr[g], 31) == cur;  // column sequences never decrease
-        if (one_segment && !diag) {
-          float s = 0.f;
-#pragma unroll
-          for (int e = 0; e < 32; ++e) s = fmaf(__uint_as_float(pv[e]), __uint_as_float(qv[e]), s);
-          run = fmaf(wseg, s, run);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int c = c0 + e, sc = __shfl_sync(0xffffffffu, csr[g], e);
-            if (sc != cur) {  // uniform across the warp
-              flush_segment(p.K, p.B, row_seq, cur, run);
-              run = 0.f;
-              cur = sc;
-              wseg = (!kSampled && row_seq == cur) ? 2.f : 1.f;
-            }
-            const float h = __uint_as_float(pv[e]) * __uint_as_float(qv[e]);
-            const float f = (!diag || c > row) ? wseg : (c == row ? 1.f : 0.f);
-            run = fmaf(f, h, run);
-          }
-        }
+        gram_group<!kSampled>(pv, qv, cs, g * 32, row, diag, rows, p.K, p.B, cur, wseg, run);
+        cs = cs_next;
       }
-      flush_segment(p.K, p.B, row_seq, cur, run);
+      flush_rows(p.K, p.B, rows, cur, run);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(accempty_bar(acc));
@@ -261,9 +224,10 @@ isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_gram<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
-  GramParams p{tokseq, K, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info, 0, 0};
+  GramParams p{tokseq, K, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info, 0, 0, 0};
   const long long units = (long long)p.nT * (p.nT + 1) / 2;
   const int grid = (int)std::min<long long>(units, sms);
+  p.strip = gram_strip_width(2.0 * kTT * (d_in + d_out), grid);
   {
     LaunchScope scope(kIdGram, st);
     k_bf16_gram<false><<<grid, kThreads, kSmemBytes, st>>>(mapX, mapY, mapX, mapY, p);
@@ -291,7 +255,7 @@ isopo_status bf16_sampled(const void* X, const void* dY, int64_t T, int d_in, in
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_gram<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   ISOPO_CUDA_TRY(cudaMemsetAsync(Mt, 0, sizeof(float) * (size_t)n_samples * B, st));
-  GramParams p{tokseq, Mt, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info, n_samples, (n_samples + kTT - 1) / kTT};
+  GramParams p{tokseq, Mt, T, B, (int)((T + kTT - 1) / kTT), d_in, d_out, info, n_samples, (n_samples + kTT - 1) / kTT, 0};
   const long long units = (long long)p.n_row_tiles * p.nT;
   const int grid = (int)std::min<long long>(units, sms);
   {
