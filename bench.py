@@ -2,7 +2,8 @@
 """Benchmark of the ISOPO per-layer hot path on B200.
 
 One "step" = the whole hot path (isopo_layer_gram -> isopo_transform_advantages -> isopo_weight_grad)
-for the seven projections of one transformer block over one ragged synthetic microbatch.  The
+for the seven projections of one transformer block over one ragged synthetic microbatch: K for every
+projection, then the coefficients of all seven in one batched transform launch, then every dW.  The
 default workload is the 1.5B-class block (d_model 1536, FFN 8960, kv 256; 256 sequences with
 log-uniform lengths in [256, 4096], ~355k tokens), the shapes the throughput target is quoted on.
 
@@ -240,39 +241,59 @@ def run_gpu(args):
     sampled = args.route == "sampled"
     # Algorithm 1 draws its overlap samples with randperm: the bench draws them once, seeded, on the host
     sample_rows = np.random.default_rng(w.seed + 17).permutation(T)[: args.samples].astype(np.int64)
+    # the stored route keeps every projection's workspace until the block's coefficients are known, so
+    # that one batched launch solves for all of them; with --transform single one workspace is reused
+    batched = not sampled and args.transform == "batched"
     layers = []
-    ws_bytes = 0
+    ws_sizes = []
     for layer in w_layers:
         X, dY = wl.layer_inputs_device(w, layer, T, dev)
         if sampled:
             path = b.PATH_GRAM
-            ws_bytes = max(ws_bytes, b.isopo_sampled_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B,
-                                                                     len(sample_rows)))
+            ws_sizes.append(b.isopo_sampled_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, len(sample_rows)))
         else:
             path = b.isopo_choose_path(dt_code, T, layer.d_in, layer.d_out, B)
-            ws_bytes = max(ws_bytes, b.isopo_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, path))
+            ws_sizes.append(b.isopo_workspace_bytes(dt_code, T, layer.d_in, layer.d_out, B, path))
         layers.append({"layer": layer, "X": X, "dY": dY, "path": path,
                        "K": torch.empty((B, B), dtype=torch.float32, device=dev),
                        "c": torch.empty(B, dtype=torch.float32, device=dev),
                        "dW": torch.zeros((layer.d_out, layer.d_in), dtype=torch.float32, device=dev),
                        "lam": 0.0})
-    raw = torch.empty(ws_bytes + 1024, dtype=torch.uint8, device=dev)
-    shift = (-raw.data_ptr()) % 1024
-    ws = raw[shift:shift + ws_bytes]
+
+    def aligned(nbytes):
+        raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        shift = (-raw.data_ptr()) % 1024
+        return raw[shift:shift + nbytes]
+
+    if batched:
+        for L, n in zip(layers, ws_sizes):
+            L["ws"] = aligned(n)
+    else:
+        shared_ws = aligned(max(ws_sizes))
+        for L in layers:
+            L["ws"] = shared_ws
     A = torch.from_numpy(A_host).to(dev)
     info = torch.zeros(1, dtype=torch.int32, device=dev)
 
     def layer_calls(L):
         if sampled:  # Algorithm 1: coefficients from sampled token rows, then the folded weight-gradient GEMM
-            b.isopo_sampled_coefficients(L["X"], L["dY"], off, sample_rows, A, L["lam"], L["c"], ws, info, L["F2"])
+            b.isopo_sampled_coefficients(L["X"], L["dY"], off, sample_rows, A, L["lam"], L["c"], L["ws"], info, L["F2"])
         else:
-            b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], ws, info, L["path"])
+            b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], L["ws"], info, L["path"])
             b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
-        b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], ws, info, L["path"], 0.0)
+        b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], L["ws"], info, L["path"], 0.0)
 
     def step():
+        if not batched:
+            for L in layers:
+                layer_calls(L)
+            return
         for L in layers:
-            layer_calls(L)
+            b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], L["ws"], info, L["path"])
+        b.isopo_transform_advantages_batched([L["K"] for L in layers], A, variant, [L["lam"] for L in layers],
+                                             [L["c"] for L in layers], info)
+        for L in layers:
+            b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], L["ws"], info, L["path"], 0.0)
 
     # the regulariser is an absolute number the caller carries from earlier minibatches:
     # 1e-3 * mean(diag K) (stored route) or 1e-3 * mean(F^2) (sampled route), taken once from an untimed pass
@@ -458,8 +479,10 @@ def run_gpu(args):
                    "layers": [f"{L['layer'].name}:{L['layer'].d_in}->{L['layer'].d_out}" for L in layers],
                    "paths": ["gram" if L["path"] == b.PATH_GRAM else "materialise" for L in layers],
                    "l2": "inputs larger than L2 (no flush needed)",
-                   "step": ("sampled_coefficients + weight_grad" if sampled else
-                            "layer_gram + transform_advantages + weight_grad") + " for each projection"},
+                   "step": ("sampled_coefficients + weight_grad for each projection" if sampled else
+                            "layer_gram for each projection, one transform_advantages_batched for all, weight_grad "
+                            "for each projection" if batched else
+                            "layer_gram + transform_advantages + weight_grad for each projection")},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(sum(v[1] for v in prof.values())),
@@ -489,6 +512,9 @@ def main():
                     help="stored: K from materialised per-sequence gradients (both variants); sampled: Algorithm 1's "
                          "token-sampled Fisher norm + folded weight-gradient GEMM (non-interacting variant)")
     ap.add_argument("--samples", type=int, default=128, help="n_overlap_samples of the sampled route")
+    ap.add_argument("--transform", default="batched", choices=["batched", "single"],
+                    help="stored route: batched = every projection keeps its workspace and one launch solves for all "
+                         "their coefficients; single = one call per projection, one shared workspace")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--layers", default="", help="comma-separated projection names (default: all of the block)")

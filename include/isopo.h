@@ -169,6 +169,28 @@ ISOPO_API isopo_status isopo_transform_advantages_rel(const float* K, const floa
                                                       float* coeffs, int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_transform_advantages_batched: the transform for several layers of one microbatch in ONE
+ * launch (layer l on its own CTA, so the layers' solves run side by side instead of one after the
+ * other).  The interacting solve of Alg. 2 is a single-CTA, latency-bound computation; a caller that keeps
+ * the K of several projections (e.g. the seven of a transformer block) before asking for their
+ * coefficients pays for one solve instead of n_layers.  All layers share A, B and the variant.
+ *
+ *   n_layers  1 .. ISOPO_MAX_BATCH
+ *   K         HOST array of n_layers device pointers, each float32 [B, B] as for isopo_transform_advantages
+ *   lambda    HOST array of n_layers regularisers (>= 0): absolute if states == NULL, else factors of
+ *             the running means as in isopo_transform_advantages_rel (GENERAL: ignored either way,
+ *             opt_pqr_regs holds the three absolute regularisers or factors for all layers)
+ *   states    NULL, or HOST array of n_layers device pointers to float32 [4] running-mean states
+ *   coeffs    HOST array of n_layers device pointers, each float32 [B], overwritten
+ * The host arrays are read before the call returns.  A non-positive pivot k of layer l is reported
+ * as *info = k + (l << 16) (the first one found wins).  Results are those of n_layers single calls.
+ */
+ISOPO_API isopo_status isopo_transform_advantages_batched(int n_layers, const float* const* K, const float* A, int B,
+                                                          isopo_variant variant, const float* lambda,
+                                                          const float* opt_pqr_regs, const float* const* states,
+                                                          float* const* coeffs, int32_t* info, void* cuda_stream);
+
+/*
  * isopo_weight_grad: dW = beta * dW + sum_i coeffs[i] * G_i   (Alg. 1 "grad += advantages * rescaled
  * gradient" and "mod.grad += grad"; Alg. 2 "stack(seq_grads) @ advantages_preconditioned").
  *
@@ -212,6 +234,7 @@ ISOPO_API isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dt
  * Other arguments and conventions as for isopo_layer_gram.
  */
 #define ISOPO_MAX_SAMPLES 4096
+#define ISOPO_MAX_BATCH 32
 ISOPO_API size_t isopo_sampled_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, int n_samples);
 ISOPO_API isopo_status isopo_sampled_coefficients(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in,
                                                   int d_out, const int64_t* seq_offsets_host, int B,

@@ -28,7 +28,7 @@ EXPORTS = (
     "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad",
     "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
     "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
-    "isopo_reg_ema_update", "isopo_transform_advantages_rel",
+    "isopo_reg_ema_update", "isopo_transform_advantages_rel", "isopo_transform_advantages_batched",
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
@@ -77,6 +77,9 @@ def _load():
                                                c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
     lib.isopo_reg_ema_update.restype = c.c_int
     lib.isopo_reg_ema_update.argtypes = [c.c_void_p, c.c_int, c.c_float, c.c_void_p, c.c_void_p]
+    lib.isopo_transform_advantages_batched.restype = c.c_int
+    lib.isopo_transform_advantages_batched.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_void_p,
+                                                       c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.isopo_transform_advantages_rel.restype = c.c_int
     lib.isopo_transform_advantages_rel.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
                                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -203,6 +206,35 @@ def isopo_transform_advantages_rel(K: torch.Tensor, A: torch.Tensor, variant: in
                                             g.ctypes.data if g is not None else None, state.data_ptr(),
                                             coeffs.data_ptr(), info.data_ptr(), _stream())
     _check(st, "isopo_transform_advantages_rel")
+
+
+def isopo_transform_advantages_batched(Ks, A: torch.Tensor, variant: int, lams, coeffs, info: torch.Tensor,
+                                       pqr_regs=None, states=None) -> None:
+    """One launch for the layers Ks[l] -> coeffs[l] (lists of tensors); lams are absolute regularisers, or
+    factors of the running means when `states` (a list of device float32 [4] tensors) is given."""
+    n, B = len(Ks), A.numel()
+    assert len(coeffs) == n and len(lams) == n and (states is None or len(states) == n)
+    for K, co in zip(Ks, coeffs):
+        assert K.dtype == torch.float32 and K.is_contiguous() and K.numel() == B * B
+        assert co.dtype == torch.float32 and co.is_contiguous() and co.numel() == B
+    assert A.dtype == torch.float32
+    k_ptrs = np.array([K.data_ptr() for K in Ks], dtype=np.uint64)
+    c_ptrs = np.array([co.data_ptr() for co in coeffs], dtype=np.uint64)
+    lam = np.ascontiguousarray(np.asarray(lams, dtype=np.float32))
+    s_ptrs = None
+    if states is not None:
+        for stt in states:
+            assert stt.dtype == torch.float32 and stt.numel() == 4 and stt.is_cuda
+        s_ptrs = np.array([stt.data_ptr() for stt in states], dtype=np.uint64)
+    g = None
+    if pqr_regs is not None:
+        g = np.ascontiguousarray(np.asarray(pqr_regs, dtype=np.float32))
+        assert g.shape == (6,)
+    st = lib.isopo_transform_advantages_batched(n, k_ptrs.ctypes.data, A.data_ptr(), B, variant, lam.ctypes.data,
+                                                g.ctypes.data if g is not None else None,
+                                                s_ptrs.ctypes.data if s_ptrs is not None else None,
+                                                c_ptrs.ctypes.data, info.data_ptr(), _stream())
+    _check(st, "isopo_transform_advantages_batched")
 
 
 def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, seq_offsets, dW: torch.Tensor,

@@ -261,6 +261,22 @@ isopo_status isopo_transform_advantages_rel(const float* K, const float* A, int 
   return transform(K, A, B, variant, factor, opt_pqr_factors, state, coeffs, info, (cudaStream_t)cuda_stream);
 }
 
+isopo_status isopo_transform_advantages_batched(int n_layers, const float* const* K, const float* A, int B,
+                                                isopo_variant variant, const float* lambda,
+                                                const float* opt_pqr_regs, const float* const* states,
+                                                float* const* coeffs, int32_t* info, void* cuda_stream) {
+  if (n_layers < 1 || n_layers > ISOPO_MAX_BATCH) return ISOPO_ERR_INVALID_ARG;
+  if (!K || !A || !lambda || !coeffs || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
+  if ((int)variant < 0 || (int)variant > (int)ISOPO_VAR_NORMALISED_RAW) return ISOPO_ERR_INVALID_ARG;
+  if (variant == ISOPO_VAR_GENERAL && !opt_pqr_regs) return ISOPO_ERR_INVALID_ARG;
+  if (variant == ISOPO_VAR_INTERACTING && B > 256) return ISOPO_ERR_UNSUPPORTED;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!K[l] || !coeffs[l] || !(lambda[l] >= 0.0f) || (states && !states[l])) return ISOPO_ERR_INVALID_ARG;
+  }
+  return transform_batched(n_layers, K, A, B, variant, lambda, opt_pqr_regs, states, coeffs, info,
+                           (cudaStream_t)cuda_stream);
+}
+
 isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
                                const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {

@@ -141,6 +141,9 @@ isopo_status sampled_coefficients(const void* X, const void* dY, isopo_dtype dty
 // transform (all variants)
 isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* pqr_regs_host,
                        const float* rel_state, float* coeffs, int32_t* info, cudaStream_t st);
+isopo_status transform_batched(int n, const float* const* K, const float* A, int B, isopo_variant v, const float* lambda,
+                               const float* pqr_regs_host, const float* const* rel_state, float* const* coeffs,
+                               int32_t* info, cudaStream_t st);
 isopo_status reg_ema_update(const float* K, int B, float decay, float* state, cudaStream_t st);
 
 }  // namespace isopo

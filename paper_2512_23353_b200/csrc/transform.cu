@@ -26,6 +26,15 @@ struct TransformParams {
                            // regularisers above are then factors of these (relative regularisation)
 };
 
+// One launch serves up to ISOPO_MAX_BATCH layers that share A and the variant: CTA l works on layer l.
+struct TransformBatch {
+  TransformParams common;  // K, coeffs, lambda, rel_state are taken from the arrays below
+  const float* K[ISOPO_MAX_BATCH];
+  float* coeffs[ISOPO_MAX_BATCH];
+  const float* rel_state[ISOPO_MAX_BATCH];
+  float lambda[ISOPO_MAX_BATCH];
+};
+
 
 __device__ __forceinline__ double warp_sum(double v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -207,8 +216,13 @@ __device__ long long g_phase[16];
 #define PHASE_ACC(n, t0) do {} while (0)
 #endif
 
-__global__ void __launch_bounds__(kThreads) k_transform(TransformParams P) {
+__global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ TransformBatch batch) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  TransformParams P = batch.common;
+  P.K = batch.K[blockIdx.x];
+  P.coeffs = batch.coeffs[blockIdx.x];
+  P.rel_state = batch.rel_state[blockIdx.x];
+  P.lambda = batch.lambda[blockIdx.x];
   __shared__ double s_trace, s_res;
   __shared__ int s_fail;
   const int B = P.B, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kThreads / 32;
@@ -346,7 +360,7 @@ __global__ void __launch_bounds__(kThreads) k_transform(TransformParams P) {
   }
   __syncthreads();
   if (s_fail) {
-    if (tid == 0) atomicCAS(P.info, 0, s_fail);
+    if (tid == 0) atomicCAS(P.info, 0, s_fail + ((int)blockIdx.x << 16));
     for (int i = tid; i < B; i += kThreads) P.coeffs[i] = 0.f;
     return;
   }
@@ -473,12 +487,19 @@ isopo_status reg_ema_update(const float* K, int B, float decay, float* state, cu
   return ISOPO_OK;
 }
 
-isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* g,
-                       const float* rel_state, float* coeffs, int32_t* info, cudaStream_t st) {
-  TransformParams P{};
-  P.K = K; P.A = A; P.coeffs = coeffs; P.info = info; P.B = B; P.variant = (int)v; P.lambda = lambda;
-  P.rel_state = rel_state;
+isopo_status transform_batched(int n, const float* const* K, const float* A, int B, isopo_variant v, const float* lambda,
+                               const float* g, const float* const* rel_state, float* const* coeffs, int32_t* info,
+                               cudaStream_t st) {
+  TransformBatch T{};
+  TransformParams& P = T.common;
+  P.A = A; P.info = info; P.B = B; P.variant = (int)v;
   if (v == ISOPO_VAR_GENERAL) { P.p = g[0]; P.q = g[1]; P.r = g[2]; P.reg_F = g[3]; P.reg_G = g[4]; P.reg_rel = g[5]; }
+  for (int l = 0; l < n; ++l) {
+    T.K[l] = K[l];
+    T.coeffs[l] = coeffs[l];
+    T.rel_state[l] = rel_state ? rel_state[l] : nullptr;
+    T.lambda[l] = lambda[l];
+  }
   size_t smem = 0;
   if (v == ISOPO_VAR_INTERACTING) {
     if (B > kMaxB) return ISOPO_ERR_UNSUPPORTED;
@@ -488,10 +509,15 @@ isopo_status transform(const float* K, const float* A, int B, isopo_variant v, f
   }
   {
     LaunchScope scope(kIdTransform, st);
-    k_transform<<<1, kThreads, smem, st>>>(P);
+    k_transform<<<n, kThreads, smem, st>>>(T);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
+}
+
+isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* g,
+                       const float* rel_state, float* coeffs, int32_t* info, cudaStream_t st) {
+  return transform_batched(1, &K, A, B, v, &lambda, g, rel_state ? &rel_state : nullptr, &coeffs, info, st);
 }
 
 }  // namespace isopo

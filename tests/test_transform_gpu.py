@@ -105,3 +105,74 @@ def test_relative_regulariser_runs_without_host_values(b):
                                         (g[3] * o_state[0][0], g[4] * o_state[0][1], g[5] * o_state[0][2]))
         assert rel_fro(c.cpu().numpy(), want) <= 1e-5
     assert int(info.item()) == 0
+
+
+@pytest.mark.parametrize("B,n", [(96, 7), (256, 7), (33, 32)])
+def test_batched_layers_equal_single_calls_and_the_oracle(b, B, n):
+    """One launch for n layers (different K and regulariser each, shared advantages) against the
+    oracle per layer, and bit-for-bit against n single calls (the same kernel, one CTA per layer)."""
+    A = np.random.default_rng(B).standard_normal(B).astype(np.float32)
+    Ad = torch.from_numpy(A).cuda()
+    Ks = [_gram(B, 1 + l % 4, 100 * B + l) * np.float32(1.0 + l) for l in range(n)]
+    Kd = [torch.from_numpy(K).cuda() for K in Ks]
+    lams = [float(np.float32((1e-3 if l % 2 else 0.3) * np.mean(np.diag(K)))) for l, K in enumerate(Ks)]
+    for variant, name in ((b.VAR_INTERACTING, orc.INTERACTING), (b.VAR_NORMALISED, orc.NORMALISED)):
+        info = torch.zeros(1, dtype=torch.int32, device="cuda")
+        cs = [torch.full((B,), float("nan"), device="cuda") for _ in range(n)]
+        b.isopo_transform_advantages_batched(Kd, Ad, variant, lams, cs, info)
+        singles = [torch.empty(B, device="cuda") for _ in range(n)]
+        for l in range(n):
+            b.isopo_transform_advantages(Kd[l], Ad, variant, lams[l], singles[l], info)
+        torch.cuda.synchronize()
+        assert int(info.item()) == 0
+        for l in range(n):
+            assert torch.equal(cs[l], singles[l]), (name, l)
+            want = orc.transform_advantages(Ks[l].astype(np.float64), A.astype(np.float64), name, lams[l])
+            cond = np.linalg.cond(Ks[l].astype(np.float64) + lams[l] * np.eye(B)) if name == orc.INTERACTING else 1.0
+            assert rel_fro(cs[l].cpu().numpy(), want) <= max(1e-6, 1e-9 * cond), (name, l, cond)
+
+
+def test_batched_relative_regulariser_and_pivot_report(b):
+    rng = np.random.default_rng(11)
+    B, n = 40, 3
+    Ks, states, o_lams = [], [], []
+    for l in range(n):
+        M = rng.standard_normal((B, 200)) * (1.0 + l)
+        K = torch.from_numpy((M @ M.T).astype(np.float32)).cuda()
+        st = torch.zeros(4, device="cuda")
+        b.isopo_reg_ema_update(K, 0.9, st)
+        Ks.append(K)
+        states.append(st)
+        o_lams.append(orc.regulariser_means(K.double().cpu().numpy())[1])  # E[K_ii]: the interacting variant's mean
+    A = torch.from_numpy(rng.standard_normal(B).astype(np.float32)).cuda()
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cs = [torch.empty(B, device="cuda") for _ in range(n)]
+    factors = [0.5, 1.0, 0.25]
+    b.isopo_transform_advantages_batched(Ks, A, b.VAR_INTERACTING, factors, cs, info, states=states)
+    torch.cuda.synchronize()
+    assert int(info.item()) == 0
+    for l in range(n):
+        want = orc.transform_advantages(Ks[l].double().cpu().numpy(), A.double().cpu().numpy(), orc.INTERACTING,
+                                        factors[l] * o_lams[l])
+        assert rel_fro(cs[l].cpu().numpy(), want) <= 1e-5, l
+    # layer 1 is made indefinite at row 7: the report names the layer and the 1-based pivot
+    bad = Ks[1].clone()
+    bad[6, 6] = -1.0
+    b.isopo_transform_advantages_batched([Ks[0], bad, Ks[2]], A, b.VAR_INTERACTING, [0.0, 0.0, 0.0], cs, info)
+    torch.cuda.synchronize()
+    assert int(info.item()) == 7 + (1 << 16)
+    assert float(cs[1].abs().max().item()) == 0.0
+
+
+def test_batched_argument_checks(b):
+    B = 8
+    K = torch.eye(B, device="cuda")
+    A = torch.ones(B, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = torch.empty(B, device="cuda")
+    with pytest.raises(b.IsopoError):
+        b.isopo_transform_advantages_batched([K] * 33, A, b.VAR_NORMALISED, [0.1] * 33, [c] * 33, info)
+    with pytest.raises(b.IsopoError):
+        b.isopo_transform_advantages_batched([K], A, b.VAR_NORMALISED, [-1.0], [c], info)
+    with pytest.raises(b.IsopoError):
+        b.isopo_transform_advantages_batched([K], A, b.VAR_GENERAL, [0.0], [c], info)
