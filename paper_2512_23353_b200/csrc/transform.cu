@@ -47,10 +47,12 @@ __device__ __forceinline__ double warp_sum(double v) {
 // K + lambda*I is held as 32 x 32 blocks (lower block triangle, block (I,J) at slot I(I+1)/2+J),
 // every block column-major: element (r, c) at [c*32 + r], so that a warp whose lane owns row r
 // reads a block column without bank conflicts and 4 consecutive rows form one float4.
-// Per block column J:  (1) warp 0 factors the diagonal block in registers (shuffles) and inverts
-// the triangular factor;  (2) one warp per block below applies the inverse (a triangular solve
-// without divisions);  (3) one warp per trailing block does the rank-32 update with 4 x 8
-// register tiles.  The solves use the stored inverses of the diagonal blocks.
+// Per block column J:  (1) one warp per block below the diagonal solves X L_JJ^T = A_IJ by
+// substitution (lane = row), while a spare warp inverts L_JJ for the solve phase;  (2) one warp per
+// trailing block does the rank-32 update with 4 x 8 register tiles; block (J+1, J+1) is updated
+// first, by all warps together, and warp 0 then factors it in registers (shuffles), so the serial
+// pivot chain of the next column runs beside the other warps' updates instead of after them.  The triangular solves with the
+// right-hand side use the stored inverses of the diagonal blocks.
 // ---------------------------------------------------------------------------------------------
 constexpr int kNB = 32;
 constexpr int kBlk = kNB * kNB;
@@ -75,9 +77,9 @@ __device__ __forceinline__ float warp_column_sums(float (&r)[kNB]) {
 }
 
 // Factors the 32 x 32 diagonal block D (column-major, symmetric input) in place into its lower
-// Cholesky factor and writes the inverse of that factor to Inv (column-major).  One warp.
+// Cholesky factor and writes 1 / L_kk to rd[k].  One warp.
 // Returns 0, or the 1-based local index of the first non-positive pivot.
-__device__ __noinline__ int warp_factor_diag(float* __restrict__ D, float* __restrict__ Inv) {
+__device__ __noinline__ int warp_factor_diag(float* __restrict__ D, float* __restrict__ rd) {
   const int lane = threadIdx.x & 31;
   float r[kNB];
 #pragma unroll
@@ -99,34 +101,44 @@ __device__ __noinline__ int warp_factor_diag(float* __restrict__ D, float* __res
   }
 #pragma unroll
   for (int c = 0; c < kNB; ++c) D[c * kNB + lane] = c <= lane ? r[c] : 0.f;
-  __syncwarp();
-  // inverse, column sweep: lane j solves L z = e_j; after step k, z[k] = Inv[k][j] is final
+  rd[lane] = rdiag;
+  return fail;
+}
+
+// Inv = L^-1 (column-major) for the factored diagonal block D with rd[k] = 1 / L_kk.  One warp.
+// Column sweep: lane j solves L z = e_j; after step k, z[k] = Inv[k][j] is final.
+__device__ __noinline__ void warp_invert_factor(const float* __restrict__ D, const float* __restrict__ rd,
+                                                float* __restrict__ Inv) {
+  const int lane = threadIdx.x & 31;
   float z[kNB];
 #pragma unroll
   for (int i = 0; i < kNB; ++i) z[i] = i == lane ? 1.f : 0.f;
 #pragma unroll
   for (int k = 0; k < kNB; ++k) {
-    z[k] *= __shfl_sync(0xffffffffu, rdiag, k);
+    z[k] *= rd[k];
 #pragma unroll
     for (int i = k + 1; i < kNB; ++i) z[i] = fmaf(-D[k * kNB + i], z[k], z[i]);  // L[i][k], broadcast
   }
 #pragma unroll
   for (int i = 0; i < kNB; ++i) Inv[lane * kNB + i] = z[i];
-  return fail;
 }
 
-// X = A * Inv^T for one 32 x 32 block A (in place); lane owns a row.  Inv lower triangular.
-__device__ __noinline__ void warp_apply_inverse(float* __restrict__ A, const float* __restrict__ Inv) {
+// X L^T = A for one 32 x 32 block A (in place); lane owns a row.  L: factored diagonal block,
+// rd[k] = 1 / L_kk.  Column k of X is final after step k and is eliminated from the later columns.
+__device__ __noinline__ void warp_solve_panel(float* __restrict__ A, const float* __restrict__ L,
+                                              const float* __restrict__ rd) {
   const int lane = threadIdx.x & 31;
-  float a[kNB], x[kNB];
+  float a[kNB];
 #pragma unroll
-  for (int c = 0; c < kNB; ++c) { a[c] = A[c * kNB + lane]; x[c] = 0.f; }
+  for (int c = 0; c < kNB; ++c) a[c] = A[c * kNB + lane];
 #pragma unroll
-  for (int p = 0; p < kNB; ++p)
+  for (int k = 0; k < kNB; ++k) {
+    a[k] *= rd[k];
 #pragma unroll
-    for (int k = p; k < kNB; ++k) x[k] = fmaf(a[p], Inv[p * kNB + k], x[k]);  // Inv[k][p], broadcast
+    for (int j = k + 1; j < kNB; ++j) a[j] = fmaf(-a[k], L[k * kNB + j], a[j]);  // L[j][k], broadcast
+  }
 #pragma unroll
-  for (int c = 0; c < kNB; ++c) A[c * kNB + lane] = x[c];
+  for (int c = 0; c < kNB; ++c) A[c * kNB + lane] = a[c];
 }
 
 // C -= A * Bm^T for 32 x 32 blocks (all column-major); lane computes a 4 x 8 sub-tile.
@@ -293,6 +305,7 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
   float* InvD = Lb + (size_t)(nb * (nb + 1) / 2) * kBlk;    // nb inverse diagonal factors
   float* vec = InvD + (size_t)nb * kBlk;                    // Bp floats
   double* sol = reinterpret_cast<double*>(vec + Bp);        // Bp doubles (8-byte aligned: all counts even)
+  float* rdiag = reinterpret_cast<float*>(sol + Bp);        // Bp floats: 1 / L_kk
   if (tid == 0) s_fail = 0;
   PHASE(0);
   // load the lower block triangle.  K is symmetric, so row j of K read along i gives column j of
@@ -336,24 +349,52 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
   PHASE(1);
   long long tph = clock64();
   (void)tph;
-  for (int J = 0; J < nb; ++J) {
-    if (warp == 0) {
-      const int f = warp_factor_diag(Lb + blk_slot(J, J) * kBlk, InvD + J * kBlk);
-      if (f != 0 && lane == 0) { s_fail = J * kNB + f; }
-    }
-    __syncthreads();
-    PHASE_ACC(8, tph);
-    if (s_fail) break;
-    for (int I = J + 1 + warp; I < nb; I += nwarps) warp_apply_inverse(Lb + blk_slot(I, J) * kBlk, InvD + J * kBlk);
+  if (warp == 0) {
+    const int f = warp_factor_diag(Lb, rdiag);
+    if (f != 0 && lane == 0) s_fail = f;
+  }
+  __syncthreads();
+  PHASE_ACC(8, tph);
+  for (int J = 0; J < nb && !s_fail; ++J) {
+    const float* Ljj = Lb + blk_slot(J, J) * kBlk;
+    // panel: blocks (I, J) below the diagonal on warps 0 .. nwarps-2; the last warp inverts L_JJ
+    if (warp == nwarps - 1) warp_invert_factor(Ljj, rdiag + J * kNB, InvD + J * kBlk);
+    else
+      for (int I = J + 1 + warp; I < nb; I += nwarps - 1) warp_solve_panel(Lb + blk_slot(I, J) * kBlk, Ljj, rdiag + J * kNB);
     __syncthreads();
     PHASE_ACC(9, tph);
-    // trailing blocks (I, Kc) with I >= Kc > J, one per warp
+    // trailing blocks (I, Kc) with I >= Kc > J; t = a(a+1)/2 + rem -> I = J+1+a, Kc = J+1+rem.
+    // t = 0 is the next diagonal block: all warps update it together, then warp 0 factors it while the
+    // others work through the rest
     const int m = nb - 1 - J, ntrail = m * (m + 1) / 2;
-    for (int t = warp; t < ntrail; t += nwarps) {
-      int a = 0, rem = t;
-      while (rem > a) { rem -= a + 1; ++a; }  // t = a(a+1)/2 + rem, rem <= a
-      const int I = J + 1 + a, Kc = J + 1 + rem;
-      warp_rank32_update(Lb + blk_slot(I, Kc) * kBlk, Lb + blk_slot(I, J) * kBlk, Lb + blk_slot(Kc, J) * kBlk);
+    if (m > 0) {
+      // all warps: rank-32 update of the next diagonal block, kNB / nwarps columns each (lane = row)
+      float* Dn = Lb + blk_slot(J + 1, J + 1) * kBlk;
+      const float* Pn = Lb + blk_slot(J + 1, J) * kBlk;
+      constexpr int kColsPerWarp = kNB / (kThreads / 32);
+      float acc[kColsPerWarp];
+#pragma unroll
+      for (int c = 0; c < kColsPerWarp; ++c) acc[c] = Dn[(warp * kColsPerWarp + c) * kNB + lane];
+#pragma unroll 8
+      for (int p = 0; p < kNB; ++p) {
+        const float a = Pn[p * kNB + lane];
+#pragma unroll
+        for (int c = 0; c < kColsPerWarp; ++c) acc[c] = fmaf(-a, Pn[p * kNB + warp * kColsPerWarp + c], acc[c]);
+      }
+#pragma unroll
+      for (int c = 0; c < kColsPerWarp; ++c) Dn[(warp * kColsPerWarp + c) * kNB + lane] = acc[c];
+      __syncthreads();
+      if (warp == 0) {
+        const int f = warp_factor_diag(Dn, rdiag + (J + 1) * kNB);
+        if (f != 0 && lane == 0) s_fail = (J + 1) * kNB + f;
+      } else {
+        for (int t = warp; t < ntrail; t += nwarps - 1) {
+          int a = 0, rem = t;
+          while (rem > a) { rem -= a + 1; ++a; }
+          const int I = J + 1 + a, Kc = J + 1 + rem;
+          warp_rank32_update(Lb + blk_slot(I, Kc) * kBlk, Lb + blk_slot(I, J) * kBlk, Lb + blk_slot(Kc, J) * kBlk);
+        }
+      }
     }
     __syncthreads();
     PHASE_ACC(10, tph);
@@ -504,7 +545,7 @@ isopo_status transform_batched(int n, const float* const* K, const float* A, int
   if (v == ISOPO_VAR_INTERACTING) {
     if (B > kMaxB) return ISOPO_ERR_UNSUPPORTED;
     const size_t nb = (size_t)(B + kNB - 1) / kNB;
-    smem = sizeof(float) * ((nb * (nb + 1) / 2 + nb) * kBlk + nb * kNB) + sizeof(double) * nb * kNB;
+    smem = sizeof(float) * ((nb * (nb + 1) / 2 + nb) * kBlk + 2 * nb * kNB) + sizeof(double) * nb * kNB;
     ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_transform, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   }
   {
