@@ -395,7 +395,9 @@ def run_gpu(args):
         roofline = {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": None, "traffic": None, "avg_launch_ms": ms_total / n, "launches": n}
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items()}
-    g_bytes = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers)  # one pass over the stored gradients
+    # one pass over the stored gradients (layers on the stored route only)
+    g_bytes = sum(2.0 * B * L["layer"].d_in * L["layer"].d_out for L in layers
+                  if not sampled and L["path"] != b.PATH_GRAM)
     for name in ("k_bf16_ntk", "k_bf16_combine"):
         if name in kernels and kernels[name]["ms_per_step"] > 0:
             kernels[name]["hbm_gbs"] = g_bytes / (kernels[name]["ms_per_step"] * 1e-3) / 1e9

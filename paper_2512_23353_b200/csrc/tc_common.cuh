@@ -45,9 +45,10 @@ isopo_status make_map_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows,
                               uint32_t box_cols, uint32_t box_rows);
 
 // Stored per-sequence gradients viewed as (x = element inside a 256-element piece row, y = sequence,
-// z = piece): boxes of 64 elements x `box_rows` sequences x 1 piece, 128-byte swizzle.  Sequences
-// past B read as zero.
-isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows);
+// z = piece): boxes of 64 elements x `box_rows` sequences x `box_pieces` pieces, 128-byte swizzle.  Sequences
+// past B and pieces past the last read as zero.
+isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows,
+                                  uint32_t box_pieces);
 
 // ---------------------------------------------------------------------------------------------
 // device: generic helpers

@@ -48,16 +48,19 @@ isopo_status make_map_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows,
   return ISOPO_OK;
 }
 
-isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows) {
+isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows,
+                                  uint32_t box_pieces) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) {
     set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
     return ISOPO_ERR_CUDA;
   }
-  if (box_rows == 0 || box_rows > 256 || ((uintptr_t)base & 15) || B == 0 || pieces == 0) return ISOPO_ERR_INVALID_ARG;
+  if (box_rows == 0 || box_rows > 256 || box_pieces == 0 || box_pieces > 256 || ((uintptr_t)base & 15) || B == 0 ||
+      pieces == 0)
+    return ISOPO_ERR_INVALID_ARG;
   cuuint64_t dims[3] = {256, B, pieces};
   cuuint64_t strides[2] = {512, B * 512};
-  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t box[3] = {64, box_rows, box_pieces};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -7,6 +7,15 @@
 // then rows 128..255 against rows 128..255 (the lower-left block is the mirror of the upper-right).
 // The float32 accumulators stay in tensor memory for the whole slab and are added into K once, with
 // reductions across CTAs by float atomics; a last tiny kernel mirrors the upper triangle.
+// For B <= 128 a box holds only the rows that exist (32, 64 or 128 >= B) but spans 8, 4 or 2 pieces, so
+// that every TMA copy still moves 32 KB (small boxes cost a fixed ~100 clocks each) and the stage is
+// again 256 rows: rows 0..127 and rows 128..255 each go through ONE 128 x 128 MMA per 16 elements,
+// which multiplies 4, 2 or 1 pieces at once.  Only the diagonal blocks of that product (a piece
+// against itself) are wanted; the epilogue adds them into K and skips the cross-piece blocks.  The
+// tensor pipe does up to four times the needed work this way, but in a quarter of the instructions:
+// with one 128 x 64 MMA per piece the pass was bound by the MMA issue rate (4.0 TB/s at B = 64
+// against 5.4 TB/s at B = 256 on the same clock), and the pipe has time to spare in an HBM-bound pass.
+// The order of the blocks inside the long contraction does not matter.
 //
 // k_bf16_combine: pure streaming, one 16-byte slot of every G_i per thread; a warp reads 512
 // contiguous bytes per sequence and the B sequences of a piece back to back.
@@ -28,8 +37,10 @@ constexpr uint32_t kTmemCols = 512;
 struct NtkParams {
   float* K;
   int B;
-  long long nkb;  // 64-element blocks in the contraction dimension
+  long long nkb;  // boxes in the contraction dimension: ceil(pieces / ppb) * 4
   int32_t* info;
+  int box_rows;   // rows of a piece inside a box: 32, 64, 128 or 256, >= B
+  int ppb;        // pieces per box = 256 / box_rows
 };
 
 __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant__ CUtensorMap mapG, NtkParams p) {
@@ -60,11 +71,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
   // this CTA's slab of the contraction dimension
   const long long per = (p.nkb + gridDim.x - 1) / gridDim.x;
   const long long kb0 = (long long)blockIdx.x * per, kb1 = min(p.nkb, kb0 + per);
-  const bool two = p.B > 128;                       // second row block present
-  const int rows = two ? 256 : 128;                 // rows per box (rows >= B arrive as zeros)
-  const uint32_t stage_tx = (uint32_t)rows * 128u;
-  const int n1 = two ? 256 : max(16, (p.B + 15) & ~15);
-  const int n2 = two ? max(16, (p.B - 128 + 15) & ~15) : 0;
+  const bool two = p.B > 128;                       // one piece per box, K in two row blocks
+  const uint32_t stage_tx = kStageBytes;            // rows >= B and pieces past the end arrive as zeros and count
+  // MMA 1: rows 0..127 against n1 rows from row 0; MMA 2: rows 128..255 against n2 rows from row 128
+  const int n1 = two ? 256 : (p.box_rows == 128 ? max(16, (p.B + 15) & ~15) : 128);
+  const int n2 = two ? max(16, (p.B - 128 + 15) & ~15) : n1;
 
   if (kb0 < kb1) {
     if (warp == 0) {
@@ -75,14 +86,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
         for (long long kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdNtk)) break;
           mbar_arrive_expect_tx(full_bar(stage), stage_tx);
-          tma_load_3d(smem_base + stage * kStageBytes, &mapG, (int)(kb & 3) * kKB, 0, (int)(kb >> 2), full_bar(stage));
+          tma_load_3d(smem_base + stage * kStageBytes, &mapG, (int)(kb & 3) * kKB, 0, (int)(kb >> 2) * p.ppb, full_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     } else if (warp == 1) {
       if (elect_one()) {  // elected, not "lane 0": lets the compiler keep the MMA operands in uniform registers
         const uint32_t idesc1 = make_idesc_bf16(128, n1, false, false);
-        const uint32_t idesc2 = make_idesc_bf16(128, two ? n2 : 16, false, false);
+        const uint32_t idesc2 = make_idesc_bf16(128, n2, false, false);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -94,11 +105,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
           for (int k16 = 0; k16 < kKB / 16; ++k16) {
             const bool accum = (kb > kb0) || k16 > 0;
             const uint64_t d0 = make_sdesc_sw128(base + k16 * 32, 16, 1024);
+            const uint64_t d1 = make_sdesc_sw128(base + 128 * 128 + k16 * 32, 16, 1024);
             mma_bf16(tmem_base, d0, d0, idesc1, accum);
-            if (two) {
-              const uint64_t d1 = make_sdesc_sw128(base + 128 * 128 + k16 * 32, 16, 1024);
-              mma_bf16(tmem_base + 256, d1, d1, idesc2, accum);
-            }
+            mma_bf16(tmem_base + 256, d1, d1, idesc2, accum);
           }
           mma_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -108,24 +117,26 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
     } else {
       const int q = warp & 3;
       const int r = q * 32 + lane;
-      if (mbar_wait(accfull_bar, 0, abort_flag, p.info, kIdNtk)) {
+      // `ok` is false only after a wait ran out; every thread still reaches the named barrier below
+      const bool ok = mbar_wait(accfull_bar, 0, abort_flag, p.info, kIdNtk);
+      {
         tc_fence_after_sync();
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
-        // block A: rows 0..127 x columns 0..n1-1 of K; keep the upper triangle c >= r
-        for (int c0 = 0; c0 < n1; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem_base + tlane + c0, v);
-          tmem_ld_wait();
-          if (r < p.B) {
+        if (two && ok) {
+          // block A: rows 0..127 x columns 0..255 of K; keep the upper triangle c >= r
+          for (int c0 = 0; c0 < n1; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_base + tlane + c0, v);
+            tmem_ld_wait();
+            if (r < p.B) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const int c = c0 + e;
-              if (c >= r && c < p.B) atomicAdd(&p.K[(size_t)r * p.B + c], __uint_as_float(v[e]));
+              for (int e = 0; e < 32; ++e) {
+                const int c = c0 + e;
+                if (c >= r && c < p.B) atomicAdd(&p.K[(size_t)r * p.B + c], __uint_as_float(v[e]));
+              }
             }
           }
-        }
-        // block B: rows 128..255 x columns 128..255
-        if (two) {
+          // block B: rows 128..255 x columns 128..255
           const int rr = 128 + r;
           for (int c0 = 0; c0 < n2; c0 += 32) {
             uint32_t v[32];
@@ -137,6 +148,36 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
                 const int c = 128 + c0 + e;
                 if (c >= rr && c < p.B) atomicAdd(&p.K[(size_t)rr * p.B + c], __uint_as_float(v[e]));
               }
+            }
+          }
+        } else if (!two) {
+          // both accumulators hold 128 / box_rows pieces side by side: row r is sequence r mod box_rows of
+          // piece-group g = r / box_rows, whose columns start at g * box_rows.  Every thread leaves the sum
+          // of its two accumulator rows in shared memory (the ring is idle by now); then the 128 threads
+          // walk the box_rows x box_rows block together, add the groups and update K.
+          const int lr = 31 - __clz(p.box_rows), rows = 1 << lr;  // box_rows is a power of two
+          const int seq = r & (rows - 1), g = r >> lr, coff = r - seq, ngroups = 128 >> lr;
+          const int ncol = min(rows, p.B);
+          float* red = reinterpret_cast<float*>(smem);  // [group][column][sequence]
+          if (ok) {
+            for (int c0 = 0; c0 < ncol; c0 += 32) {
+              uint32_t v0[32], v1[32];
+              tmem_ld32(tmem_base + tlane + coff + c0, v0);
+              tmem_ld32(tmem_base + tlane + 256 + coff + c0, v1);
+              tmem_ld_wait();
+              float* dst = red + ((((g << lr) + c0) << lr) + seq);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) dst[e << lr] = __uint_as_float(v0[e]) + __uint_as_float(v1[e]);
+            }
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps
+          if (ok) {
+            for (int idx = r; idx < (ncol << lr); idx += 128) {
+              const int sq = idx & (rows - 1), c = idx >> lr;
+              if (c < sq || sq >= p.B) continue;  // upper triangle of the sequences that exist
+              float sum = 0.f;
+              for (int h = 0; h < ngroups; ++h) sum += red[(((h << lr) + c) << lr) + sq];
+              atomicAdd(&p.K[(size_t)sq * p.B + c], sum);
             }
           }
         }
@@ -218,15 +259,16 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ 
 isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t* info, cudaStream_t st) {
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
   CUtensorMap mapG;
-  const uint32_t rows = B > 128 ? 256 : 128;
-  isopo_status s = make_map_pieces_bf16(&mapG, G, (uint64_t)B, (uint64_t)(L.n_pad / kPieceElems), rows);
+  const uint32_t rows = B > 128 ? 256 : B > 64 ? 128 : B > 32 ? 64 : 32, ppb = 256 / rows;
+  const long long pieces = L.n_pad / kPieceElems;
+  isopo_status s = make_map_pieces_bf16(&mapG, G, (uint64_t)B, (uint64_t)pieces, rows, ppb);
   if (s != ISOPO_OK) return s;
   int dev = 0, sms = 0;
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_ntk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
-  NtkParams p{K, B, L.n_pad / kKB, info};
+  NtkParams p{K, B, (pieces + ppb - 1) / ppb * 4, info, (int)rows, (int)ppb};
   const int grid = (int)std::max<long long>(1, std::min<long long>(sms, p.nkb / 8));
   {
     LaunchScope scope(kIdNtk, st);
