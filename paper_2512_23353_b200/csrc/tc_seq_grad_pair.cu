@@ -58,7 +58,21 @@ struct PairParams {
   int B, tiles_m, tiles_n;  // stored 128 x 256 tiles per gradient
   int ptiles_m;             // pair tiles along d_out = ceil(tiles_m / 2)
   int32_t* info;
+  int group_m;              // pair-tile rows per group of the tile order
 };
+
+// The pair tiles of one sequence are visited in groups of `group_m` rows, row index fastest inside a
+// group: the ~74 pairs then work on about group_m row blocks of dY and 74 / group_m column blocks of X
+// of the same tokens at a time, and what they stream stays in the L2.  Row by row instead, a layer
+// with a wide input (74 column blocks) has a whole sequence of X in flight, more than the L2 holds,
+// and reads it from HBM once per row of tiles.
+__device__ __forceinline__ void pair_tile(int pt, const PairParams& p, int& ptm, int& tn) {
+  const int per_group = p.group_m * p.tiles_n;
+  const int first = (pt / per_group) * p.group_m, in_group = pt % per_group;
+  const int gm = min(p.group_m, p.ptiles_m - first);
+  ptm = first + in_group % gm;
+  tn = in_group / gm;
+}
 
 // Shape of one unit's token loop, identical in every role.
 struct UnitShape {
@@ -141,7 +155,8 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
       bool ok = true;
       for (long long u = pair_id; u < total_units && ok; u += npairs) {
         const int k = (int)(u / ptiles), pt = (int)(u % ptiles);
-        const int ptm = pt / p.tiles_n, tn = pt % p.tiles_n;
+        int ptm, tn;
+        pair_tile(pt, p, ptm, tn);
         const int64_t t0 = s_first[k];
         const UnitShape us = unit_shape(s_len[k]);
         const int ycol = (2 * ptm + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
@@ -210,7 +225,9 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
     uint32_t acc_phase = 0;
     for (long long u = pair_id; u < total_units; u += npairs) {
       const int i = s_seq[u / ptiles], pt = (int)(u % ptiles);
-      const int tm = 2 * (pt / p.tiles_n) + (int)rank, tn = pt % p.tiles_n;
+      int ptm, tn;
+      pair_tile(pt, p, ptm, tn);
+      const int tm = 2 * ptm + (int)rank;
       const int tile = tm * p.tiles_n + tn;
       if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
       tc_fence_after_sync();
@@ -318,6 +335,9 @@ isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_
     resident_pairs[dev] = std::min(n, sms / 2);
   }
   const int npairs = (int)std::max<long long>(1, std::min<long long>(units, resident_pairs[dev]));
+  int g = 1;
+  while ((g + 1) * (g + 1) <= npairs) ++g;  // about sqrt(npairs) rows by sqrt(npairs) columns of tiles in flight
+  p.group_m = std::max(1, std::min(g, p.ptiles_m));
   {
     LaunchScope scope(kIdSeqGrad, st);
     k_bf16_seq_grad_pair<<<2 * npairs, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
