@@ -150,3 +150,28 @@ def test_ragged_tails_many_short_sequences(b, seed):
     assert np.max(np.abs(d - d_o) / d_o) <= TOL
     c_o = orc.transform_advantages(K_o, to_f64(A), orc.NORMALISED, 0.0)
     assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
+
+
+@pytest.mark.parametrize("B", [2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256])
+def test_stored_route_at_every_box_shape(b, B):
+    """The K pass packs 8, 4, 2 or 1 stored pieces into one 256-row stage according to B (<= 32, <= 64,
+    <= 128, else) and sums the pieces' diagonal blocks in its epilogue: every B around those limits,
+    on a layer of several tiles with a ragged edge (320 x 200), correlated inputs so that the
+    off-diagonal entries of K carry weight."""
+    rng = np.random.default_rng(9000 + B)
+    Ls = rng.integers(1, 6, size=B).tolist()
+    X, dY, off, A = _inputs(Ls, 320, 200, 9100 + B, correlated=True)
+    G = orc.sequence_gradients(to_f64(X), to_f64(dY), off)
+    K_o = orc.ntk(G)
+    lam = 1e-2 * float(np.mean(np.diag(K_o)))
+    res = b.isopo_layer(X, dY, off, A, b.VAR_NORMALISED, lam, b.PATH_MATERIALISE)
+    assert res.info == 0
+    K = res.K.cpu().numpy()
+    assert np.array_equal(K, K.T)
+    assert rel_fro(K, K_o) <= TOL
+    assert offdiag_rel_fro(K, K_o) <= TOL
+    d, d_o = np.diag(K), np.diag(K_o)
+    assert np.max(np.abs(d - d_o) / d_o) <= TOL
+    c_o = orc.transform_advantages(K_o, to_f64(A), orc.NORMALISED, lam)
+    assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL
+    assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
