@@ -458,21 +458,45 @@ def run_gpu(args):
         h2d = sum(L["X"].numel() * L["X"].element_size() + L["dY"].numel() * L["dY"].element_size() for L in layers)
         d2h = sum(L["dW"].numel() * 4 for L in layers)
 
+        # three streams: host -> device copies run ahead of the compute stream, results leave behind it;
+        # events order every buffer's reuse (a layer's inputs are not overwritten before the previous
+        # step's kernels on them are done, its dW not before the previous copy-out has left)
+        comp = torch.cuda.current_stream()
+        copy_s, out_s = torch.cuda.Stream(), torch.cuda.Stream()
+        ready = {id(L): torch.cuda.Event() for L in layers}
+        done = {id(L): torch.cuda.Event() for L in layers}
+        left = {id(L): torch.cuda.Event() for L in layers}
+        for L in layers:
+            done[id(L)].record(comp)
+            left[id(L)].record(comp)
+
         def e2e_step():
             for L in layers:
-                L["X"].copy_(pinned[("X", L["layer"].d_in)], non_blocking=True)
-                L["dY"].copy_(pinned[("dY", L["layer"].d_out)], non_blocking=True)
+                with torch.cuda.stream(copy_s):
+                    copy_s.wait_event(done[id(L)])
+                    L["X"].copy_(pinned[("X", L["layer"].d_in)], non_blocking=True)
+                    L["dY"].copy_(pinned[("dY", L["layer"].d_out)], non_blocking=True)
+                    ready[id(L)].record(copy_s)
+                comp.wait_event(ready[id(L)])
+                comp.wait_event(left[id(L)])
                 layer_calls(L)
-                dW_host[id(L)].copy_(L["dW"], non_blocking=True)
+                done[id(L)].record(comp)
+                with torch.cuda.stream(out_s):
+                    out_s.wait_event(done[id(L)])
+                    dW_host[id(L)].copy_(L["dW"], non_blocking=True)
+                    left[id(L)].record(out_s)
 
         e2e_step()
         torch.cuda.synchronize()
         n_e2e = max(1, min(args.steps, 3))
         a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
+        a.record(comp)
+        copy_s.wait_event(a)
         for _ in range(n_e2e):
             e2e_step()
-        c.record()
+        for L in layers:
+            comp.wait_event(left[id(L)])  # the last results have reached the host
+        c.record(comp)
         torch.cuda.synchronize()
         e2e_ms = a.elapsed_time(c) / n_e2e
         e2e = {"value": T / (e2e_ms / 1000.0), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
