@@ -175,3 +175,28 @@ def test_stored_route_at_every_box_shape(b, B):
     c_o = orc.transform_advantages(K_o, to_f64(A), orc.NORMALISED, lam)
     assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL
     assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
+
+
+def test_more_than_256_sequences_take_the_gram_route(b):
+    """The stored-gradient kernels keep all B rows of a piece on chip and stop at B = 256; beyond that
+    AUTO resolves to the Gram route and an explicit MATERIALISE request is refused.  400 sequences of
+    1..40 tokens, simple variant (the interacting solve is limited to 256 as well)."""
+    rng = np.random.default_rng(77)
+    Ls = rng.integers(1, 41, size=400).tolist()
+    X, dY, off, A = _inputs(Ls, 192, 136, 7700, correlated=True)
+    assert b.isopo_choose_path(b.BF16, int(off[-1]), 192, 136, 400) == b.PATH_GRAM
+    G = orc.sequence_gradients(to_f64(X), to_f64(dY), off)
+    K_o = orc.ntk(G)
+    lam = 1e-2 * float(np.mean(np.diag(K_o)))
+    res = b.isopo_layer(X, dY, off, A, b.VAR_NORMALISED, lam, b.PATH_AUTO)
+    assert res.info == 0
+    K = res.K.cpu().numpy()
+    assert np.array_equal(K, K.T)
+    assert rel_fro(K, K_o) <= TOL and offdiag_rel_fro(K, K_o) <= TOL
+    c_o = orc.transform_advantages(K_o, to_f64(A), orc.NORMALISED, lam)
+    assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL
+    assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
+    with pytest.raises(b.IsopoError):
+        b.isopo_layer(X, dY, off, A, b.VAR_NORMALISED, lam, b.PATH_MATERIALISE)
+    with pytest.raises(b.IsopoError):
+        b.isopo_layer(X, dY, off, A, b.VAR_INTERACTING, lam, b.PATH_AUTO)
