@@ -243,8 +243,8 @@ def run_gpu(args):
     # Algorithm 1 draws its overlap samples with randperm: the bench draws them once, seeded, on the host
     sample_rows = np.random.default_rng(w.seed + 17).permutation(T)[: args.samples].astype(np.int64)
     # the stored route keeps every projection's workspace until the block's coefficients are known, so
-    # that one batched launch solves for all of them; with --transform single one workspace is reused
-    batched = not sampled and args.transform == "batched"
+    # that one batched launch solves for all of them; with --schedule single one workspace is reused
+    batched = not sampled and args.schedule == "batched"
     layers = []
     ws_sizes = []
     for layer in w_layers:
@@ -524,6 +524,7 @@ def run_gpu(args):
                    "step": ("sampled_coefficients + weight_grad for each projection" if sampled else
                             "layer_gram for each projection, one transform_advantages_batched for all, weight_grad "
                             "for each projection" if batched else
+
                             "layer_gram + transform_advantages + weight_grad for each projection")},
         "clocks": clocks,
         "e2e": e2e,
@@ -554,7 +555,7 @@ def main():
                     help="stored: K from materialised per-sequence gradients (both variants); sampled: Algorithm 1's "
                          "token-sampled Fisher norm + folded weight-gradient GEMM (non-interacting variant)")
     ap.add_argument("--samples", type=int, default=128, help="n_overlap_samples of the sampled route")
-    ap.add_argument("--transform", default="batched", choices=["batched", "single"],
+    ap.add_argument("--schedule", default="batched", choices=["batched", "single"],
                     help="stored route: batched = every projection keeps its workspace and one launch solves for all "
                          "their coefficients; single = one call per projection, one shared workspace")
     ap.add_argument("--skip-e2e", action="store_true")
