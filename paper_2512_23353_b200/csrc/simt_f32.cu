@@ -50,6 +50,28 @@ __global__ void k_tokscale(const int64_t* __restrict__ off, int B, int64_t T, co
   }
 }
 
+// k_store_offsets + k_tokseq / k_tokscale in one launch when all B + 1 offsets fit one argument block:
+// every CTA copies them to shared memory and searches there; CTA 0 also leaves them in the workspace.
+template <bool kScale>
+__global__ void __launch_bounds__(256) k_prep_small(OffsetArgs a, int B, int64_t T, int64_t* __restrict__ off_dev,
+                                                    const float* __restrict__ coeffs, void* __restrict__ out) {
+  __shared__ int64_t s_off[kArgChunk];
+  for (int i = threadIdx.x; i <= B; i += blockDim.x) {
+    s_off[i] = a.v[i];
+    if (blockIdx.x == 0) off_dev[i] = a.v[i];
+  }
+  __syncthreads();
+  for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
+    int lo = 0, hi = B;  // invariant: off[lo] <= t < off[hi]
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (s_off[mid] <= t) lo = mid; else hi = mid;
+    }
+    if (kScale) static_cast<float*>(out)[t] = coeffs[lo];
+    else static_cast<int32_t*>(out)[t] = lo;
+  }
+}
+
 // Accumulates, for tokens [t0, t1), acc[4][4] += w_t * dY[t, m0+4ty+a] * X[t, n0+4tx+b].
 template <bool kScaled>
 __device__ __forceinline__ void gemm_tokens(const float* __restrict__ X, const float* __restrict__ dY, int d_in,
@@ -225,8 +247,23 @@ isopo_status store_i64(const int64_t* host, int64_t n, int64_t* dev, cudaStream_
   return ISOPO_OK;
 }
 
+template <bool kScale>
+static isopo_status launch_prep_small(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, const float* coeffs,
+                                      void* out, cudaStream_t st) {
+  OffsetArgs a;
+  for (int t = 0; t <= B; ++t) a.v[t] = off_host[t];
+  const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
+  {
+    LaunchScope scope(kIdPrep, st);
+    k_prep_small<kScale><<<grid, 256, 0, st>>>(a, B, T, off_dev, coeffs, out);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
 isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, int32_t* tokseq,
                          cudaStream_t st) {
+  if (B + 1 <= kArgChunk) return launch_prep_small<false>(off_host, B, T, off_dev, nullptr, tokseq, st);
   isopo_status s = store_i64(off_host, (int64_t)B + 1, off_dev, st);
   if (s != ISOPO_OK) return s;
   const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
@@ -240,6 +277,7 @@ isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off
 
 isopo_status launch_tokscale(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, const float* coeffs,
                              float* tokscale, cudaStream_t st) {
+  if (B + 1 <= kArgChunk) return launch_prep_small<true>(off_host, B, T, off_dev, coeffs, tokscale, st);
   isopo_status s = store_i64(off_host, (int64_t)B + 1, off_dev, st);
   if (s != ISOPO_OK) return s;
   const int grid = (int)std::min<int64_t>((T + 255) / 256, 1184);
