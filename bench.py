@@ -444,6 +444,27 @@ def run_gpu(args):
         plain_ms += plain_by_layer[-1]
     overhead = ms_per_step / plain_ms
 
+    # ---- the same step replayed from a CUDA graph (launch-bound workloads): extra figure, not the metric ----
+    graph = None
+    if args.graph:
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            step()
+        for _ in range(3):
+            g.replay()
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            g.replay()
+        c.record()
+        torch.cuda.synchronize()
+        if int(info.item()) != 0:
+            raise SystemExit(f"device-side error during graph replay: info={int(info.item()):#x}")
+        graph = {"ms_per_step": a.elapsed_time(c) / args.steps, "steps": args.steps,
+                 "note": "one captured step replayed back to back; no L2 flush between replays"}
+
     # ---- end to end: host buffers, copies inside the timed region ----
     e2e = None
     if not args.skip_e2e:
@@ -528,6 +549,7 @@ def run_gpu(args):
                             "layer_gram + transform_advantages + weight_grad for each projection")},
         "clocks": clocks,
         "e2e": e2e,
+        "cuda_graph": graph,
         "gpu_launches": int(sum(v[1] for v in prof.values())),
         "roofline": roofline,
         "cpu_baseline": cpu,
@@ -558,6 +580,8 @@ def main():
     ap.add_argument("--schedule", default="batched", choices=["batched", "single"],
                     help="stored route: batched = every projection keeps its workspace and one launch solves for all "
                          "their coefficients; single = one call per projection, one shared workspace")
+    ap.add_argument("--graph", action="store_true",
+                    help="also capture one step in a CUDA graph and time its replays (reported under cuda_graph)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--layers", default="", help="comma-separated projection names (default: all of the block)")
