@@ -8,12 +8,18 @@
 // here: under the power cap the extra shared-memory traffic and the busy scaler warps cost more
 // than the extra pass over 1/6 .. 1/35 of the operand bytes.
 //
-// The GEMM is the pipeline of tc_seq_grad_pair.cu with other work units: (256 x 256 tile of dW, slab
-// of tokens), slab-major so that the pairs running at one time read the same tokens out of L2.
+// The GEMM is the pipeline of tc_seq_grad_pair.cu with other work units: (256 x 512 block of dW, slab
+// of tokens), slab-major so that the pairs running at one time read the same tokens out of L2.  The
+// block is two 256 x 256 accumulators side by side that share the dY operand: all 512 columns of
+// tensor memory, so a unit's epilogue is not overlapped, but a unit is a long token slab (there are
+// only a few per pair).  Against one 256 x 256 tile per unit this moves 3/4 of the operand bytes
+// from L2 to the SMs per flop and streams the inputs from HBM about half as often (every round of
+// units re-reads its slab, and there are half as many units per slab); under the power cap both show
+// up as clock.
 //
 //   warp 0          TMA producer; both CTAs' copies complete on the barrier in CTA 0
-//   warp 1, CTA 0   MMA issuer (one elected thread), tcgen05.mma.cta_group::2 256 x 256 x 16
-//   warps 2-5       epilogue: TMEM -> float32 red.global.add.v4 into dW (token slabs of a tile meet there)
+//   warp 1, CTA 0   MMA issuer (one elected thread), 2 x tcgen05.mma.cta_group::2 256 x 256 x 16 per step
+//   warps 2-5       epilogue: TMEM -> float32 red.global.add.v4 into dW (token slabs of a block meet there)
 //
 // Every wait is bounded; the teardown is that of tc_seq_grad_pair.cu.
 #include <algorithm>
@@ -27,22 +33,23 @@ namespace {
 using namespace tc;
 
 constexpr int kKB = 64;                              // tokens per pipeline stage
-constexpr int kStages = 6;
+constexpr int kStages = 4;
 constexpr int kHalf = 128;
-constexpr int kChunkBytes = kKB * 128;
-constexpr int kOperandBytes = 2 * kChunkBytes;
-constexpr int kStageBytes = 2 * kOperandBytes;
+constexpr int kChunkBytes = kKB * 128;           // 64 tokens x 64 columns
+constexpr int kOperandBytes = 2 * kChunkBytes;   // one CTA's 128 columns of an operand
+constexpr int kStageBytes = 3 * kOperandBytes;   // dY half, X half of the left tile, X half of the right tile
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kPairN = 256;
+constexpr int kUnitOverhead = 16;  // a unit's epilogue and pipeline fill, in 64-token stages (host cost model)
 static_assert(kSmemBytes <= 227 * 1024, "shared memory");
 
 struct FoldedPairParams {
   float* dW;
   int64_t T, slab;  // tokens per work unit (a multiple of kKB)
   int nslabs, d_in, d_out;
-  int ptiles_m, tiles_n;
+  int ptiles_m, tiles_n;  // 256-row blocks of d_out; 512-column blocks of d_in
   int32_t* info;
 };
 
@@ -69,7 +76,8 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(accfull_bar(b), 1); mbar_init(accempty_bar(b), 8); }
+    mbar_init(accfull_bar(0), 1);
+    mbar_init(accempty_bar(0), 8);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -105,17 +113,18 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
         int64_t t0;
         int nkb;
         unit_tokens(u, t0, nkb);
-        const int ycol = (2 * ptm + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
+        const int ycol = (2 * ptm + (int)rank) * kHalf, xcol = tn * 2 * kPairN + (int)rank * kHalf;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait_pair(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort, p.info, kIdWeightGrad))) break;
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kOperandBytes;
-          const int y = (int)(t0 + (int64_t)kb * kKB);  // rows past T read as zero
+          const int y = (int)(t0 + (int64_t)kb * kKB);  // rows past T and columns past d_in read as zero
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * kStageBytes);
           const uint32_t fb = full_at_leader + 8u * stage;
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             tma_load_2d_pair(a_dst + c * kChunkBytes, &mapY, ycol + c * 64, y, fb);
             tma_load_2d_pair(b_dst + c * kChunkBytes, &mapX, xcol + c * 64, y, fb);
+            tma_load_2d_pair(b_dst + kOperandBytes + c * kChunkBytes, &mapX, xcol + kPairN + c * 64, y, fb);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -125,15 +134,16 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
     // ------------------------------------------------------------------ MMA issuer (one thread of CTA 0)
     if (rank == 0 && elect_one()) {
       constexpr uint32_t idesc = make_idesc_bf16(256, kPairN, /*a_mn=*/true, /*b_mn=*/true);
-      int stage = 0, acc = 0;
+      int stage = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (long long u = pair_id; u < total_units && ok; u += npairs) {
         int64_t t0;
         int nkb;
         unit_tokens(u, t0, nkb);
-        if (!(ok = mbar_wait_pair(accempty_bar(acc), acc_phase ^ 1u, abort_flag, peer_abort, p.info, kIdWeightGrad))) break;
-        const uint32_t d_tmem = tmem_base + (uint32_t)acc * kPairN;
+        if (!(ok = mbar_wait_pair(accempty_bar(0), acc_phase ^ 1u, abort_flag, peer_abort, p.info, kIdWeightGrad))) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait_pair(full_bar(stage), phase, abort_flag, peer_abort, p.info, kIdWeightGrad))) break;
           tc_fence_after_sync();
@@ -142,14 +152,16 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
           for (int k16 = 0; k16 < kKB / 16; ++k16) {
             const uint64_t a_desc = make_sdesc_sw128(a_addr + k16 * 2048, kChunkBytes, 1024);
             const uint64_t b_desc = make_sdesc_sw128(b_addr + k16 * 2048, kChunkBytes, 1024);
+            const uint64_t b2_desc = make_sdesc_sw128(b_addr + kOperandBytes + k16 * 2048, kChunkBytes, 1024);
             mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | k16) != 0);
+            mma_bf16_pair(d_tmem + kPairN, a_desc, b2_desc, idesc, (kb | k16) != 0);
           }
           mma_commit_pair(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        mma_commit_pair(accfull_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        mma_commit_pair(accfull_bar(0));
+        acc_phase ^= 1u;
       }
     }
   } else if (warp < 6) {
@@ -157,17 +169,16 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
     const int q = warp & 3;
     const int row = q * 32 + lane;
     const uint32_t accempty_at_leader = map_to_cta(accempty_bar(0), 0);
-    int acc = 0;
     uint32_t acc_phase = 0;
     for (long long u = pair_id; u < total_units; u += npairs) {
       const int pt = (int)(u % ptiles);
-      const int m = (2 * (pt / p.tiles_n) + (int)rank) * kHalf + row, n0 = (pt % p.tiles_n) * kPairN;
-      if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdWeightGrad)) break;
+      const int m = (2 * (pt / p.tiles_n) + (int)rank) * kHalf + row, n0 = (pt % p.tiles_n) * 2 * kPairN;
+      if (!mbar_wait_pair(accfull_bar(0), acc_phase, abort_flag, peer_abort, p.info, kIdWeightGrad)) break;
       tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
       float* dst = p.dW + (size_t)m * p.d_in + n0;
 #pragma unroll 2
-      for (int jc = 0; jc < kPairN / 32; ++jc) {
+      for (int jc = 0; jc < 2 * kPairN / 32; ++jc) {
         uint32_t r[32];
         tmem_ld32(taddr + jc * 32, r);
         tmem_ld_wait();
@@ -185,8 +196,8 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive_remote(accempty_at_leader + 8u * acc);
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (lane == 0) mbar_arrive_remote(accempty_at_leader);
+      acc_phase ^= 1u;
     }
   }
 
@@ -259,13 +270,19 @@ isopo_status bf16_weight_grad_pair(const void* X, const void* dY, int64_t T, int
   FoldedPairParams p{};
   p.dW = dW; p.T = T; p.d_in = d_in; p.d_out = d_out; p.info = info;
   p.ptiles_m = ((d_out + kHalf - 1) / kHalf + 1) / 2;
-  p.tiles_n = (d_in + kPairN - 1) / kPairN;
-  // token slabs: about eight (tile, slab) units per pair so that the round-robin share is even; every
-  // slab a multiple of the stage depth.  (Slabs small enough for their rows to stay in L2 across the
-  // waves of tiles were measured slower: the float32 reductions into dW grow with the slab count.)
+  p.tiles_n = (d_in + 2 * kPairN - 1) / (2 * kPairN);
+  // token slabs: the count (up to 64) whose rounds of units take least, a round costing its slab plus the
+  // unit's exposed epilogue and pipeline fill (about kUnitOverhead stages' worth); ties go to fewer slabs.  Every slab is a multiple of the stage depth.
+  // (Slabs small enough for their rows to stay in L2 across the rounds were measured slower: the
+  // float32 reductions into dW grow with the slab count.)
   const long long ptiles = (long long)p.ptiles_m * p.tiles_n, pairs = resident_pairs[dev];
   const long long kblocks = (T + kKB - 1) / kKB;
-  long long nslabs = std::max<long long>(1, std::min<long long>(kblocks, (8 * pairs + ptiles - 1) / ptiles));
+  long long nslabs = 1, best = -1;
+  for (long long n = 1; n <= std::min<long long>(64, kblocks); ++n) {
+    const long long per = (kblocks + n - 1) / n, rounds = (ptiles * n + pairs - 1) / pairs;
+    const long long cost = rounds * (per + kUnitOverhead);
+    if (best < 0 || cost < best) { best = cost; nslabs = n; }
+  }
   const long long kb_per = (kblocks + nslabs - 1) / nslabs;
   nslabs = (kblocks + kb_per - 1) / kb_per;
   p.slab = kb_per * kKB;
