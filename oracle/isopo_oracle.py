@@ -174,6 +174,20 @@ def transform_advantages(K, A, variant, lam=0.0, pqr=None, regs=None):
     raise ValueError(f"unknown variant {variant!r}")
 
 
+def spectral_coefficients(K, A, lam=0.0, rel_cutoff=0.0):
+    """The interacting transform in the spectral form Algorithm 2 prints, with its spectrum returned:
+    K = U D U^T (symmetric eigendecomposition), preconditioner 1 / (D + lam) per eigen-direction,
+    c = U (preconditioner * (U^T A)).  Directions whose eigenvalue is not above rel_cutoff * max(D) are
+    left out of the sum (rel_cutoff = 0 and a positive definite K: every direction, i.e. the
+    interacting variant; lam = 0 with a cut-off: the pseudo-inverse on the kept range).
+    Returns (c, D sorted from the largest down)."""
+    K, A = _f64(K), _f64(A)
+    D, U = np.linalg.eigh(K)
+    keep = D > rel_cutoff * np.max(D)
+    pre = np.where(keep, 1.0 / np.where(keep, D + lam, 1.0), 0.0)
+    return U @ (pre * (U.T @ A)), D[::-1].copy()
+
+
 def regulariser_means(K):
     """Microbatch means of the quantities the relative regulariser is added to (generalised
     re-scaling figure: `reg(val) = val + regularization * expectation(val)`):

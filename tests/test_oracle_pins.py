@@ -398,6 +398,56 @@ def test_regulariser_means_and_ema():
     assert s[1] == 8
 
 
+# ----------------------------------------------------------------------------- spectral form of Algorithm 2
+
+def test_spectral_form_two_by_two_closed_form():
+    """K = [[a, b], [b, a]]: eigenvalues a + b and a - b on (1, 1)/sqrt2 and (1, -1)/sqrt2, so
+    c = (A1 + A2)/(2 (a + b + lam)) (1, 1) + (A1 - A2)/(2 (a - b + lam)) (1, -1); with the small direction
+    cut off only the first term stays."""
+    a, b, lam = 3.0, 1.0, 0.25
+    K, A = np.array([[a, b], [b, a]]), np.array([2.0, -1.0])
+    c, D = orc.spectral_coefficients(K, A, lam)
+    hi, lo = (A[0] + A[1]) / (2 * (a + b + lam)), (A[0] - A[1]) / (2 * (a - b + lam))
+    np.testing.assert_allclose(D, [a + b, a - b], rtol=1e-14)
+    np.testing.assert_allclose(c, [hi + lo, hi - lo], rtol=1e-13)
+    c_cut, _ = orc.spectral_coefficients(K, A, lam, rel_cutoff=0.6)  # 2 <= 0.6 * 4: dropped
+    np.testing.assert_allclose(c_cut, [hi, hi], rtol=1e-13)
+    c_keep, _ = orc.spectral_coefficients(K, A, lam, rel_cutoff=0.4)  # 2 > 0.4 * 4: kept
+    np.testing.assert_allclose(c_keep, c, rtol=1e-14)
+
+
+@pytest.mark.parametrize("seed", [41, 42])
+def test_spectral_form_equals_elimination_and_its_spectrum_has_the_trace_and_determinant(seed):
+    X, dY, off, A = _problem(seed, B=6)
+    K = orc.ntk(orc.sequence_gradients(X, dY, off))
+    lam = 1e-2 * np.mean(np.diag(K))
+    c, D = orc.spectral_coefficients(K, A, lam)
+    np.testing.assert_allclose(c, _gauss_solve(K + lam * np.eye(6), A), rtol=1e-9)
+    assert np.all(np.diff(D) <= 0)
+    assert np.sum(D) == pytest.approx(np.trace(K), rel=1e-12)
+    # product of the shifted eigenvalues = determinant of the shifted matrix, by elimination pivots
+    M = K + lam * np.eye(6)
+    piv = 1.0
+    M = M.copy()
+    for k in range(6):
+        piv *= M[k, k]
+        M[k + 1:] -= np.outer(M[k + 1:, k] / M[k, k], M[k])
+    assert np.prod(D + lam) == pytest.approx(piv, rel=1e-9)
+
+
+def test_spectral_form_with_cutoff_on_a_rank_deficient_kernel_is_the_pseudo_inverse():
+    """Two copies of every sequence: K has rank B/2.  With lam = 0 and the null directions cut off the
+    result is the minimum-norm solution K^+ A (numpy's pinv, computed from the SVD)."""
+    X, dY, off, A = _problem(43, B=3)
+    G = orc.sequence_gradients(X, dY, off)
+    K = orc.ntk(np.concatenate([G, G]))
+    A2 = np.concatenate([A, 0.5 * A])
+    c, D = orc.spectral_coefficients(K, A2, 0.0, rel_cutoff=1e-9)
+    assert np.sum(D > 1e-9 * D[0]) == 3
+    np.testing.assert_allclose(c, np.linalg.pinv(K, rcond=1e-9) @ A2, rtol=1e-8, atol=1e-12 * np.abs(c).max())
+    np.testing.assert_allclose(c[:3], c[3:], rtol=1e-8)  # symmetric in the copies
+
+
 def test_pins_catch_planted_mistakes(monkeypatch):
     """Each mistake planted in the oracle (an off-by-one partition, a one-sided kernel fill, a
     dropped normalisation, a wrong regulariser sign) makes a pin above fail."""
@@ -427,7 +477,27 @@ def test_pins_catch_planted_mistakes(monkeypatch):
     def sampled_transposed_samples(X, dY, off, rows):      # takes the samples' rows from the wrong end
         return true_sampled(X, dY, off, (int(np.asarray(off)[-1]) - 1) - np.asarray(rows))
 
+    true_spec = orc.spectral_coefficients
+
+    def spectral_cutoff_on_wrong_side(K, A, lam=0.0, rel_cutoff=0.0):  # keeps the small directions instead
+        K, A = np.asarray(K, float), np.asarray(A, float)
+        D, U = np.linalg.eigh(K)
+        keep = D <= rel_cutoff * np.max(D) if rel_cutoff > 0 else np.ones_like(D, bool)
+        return U @ (np.where(keep, 1.0 / (D + lam), 0.0) * (U.T @ A)), D[::-1].copy()
+
+    def spectral_untransposed(K, A, lam=0.0, rel_cutoff=0.0):          # U (pre * (U A)) instead of U^T A
+        K, A = np.asarray(K, float), np.asarray(A, float)
+        D, U = np.linalg.eigh(K)
+        return U @ ((1.0 / (D + lam)) * (U @ A)), D[::-1].copy()
+
+    def spectral_ascending(K, A, lam=0.0, rel_cutoff=0.0):             # spectrum in eigh's order
+        c, D = true_spec(K, A, lam, rel_cutoff)
+        return c, D[::-1].copy()
+
     plants = [
+        ("spectral_coefficients", spectral_cutoff_on_wrong_side, test_spectral_form_two_by_two_closed_form),
+        ("spectral_coefficients", spectral_untransposed, lambda: test_spectral_form_equals_elimination_and_its_spectrum_has_the_trace_and_determinant(41)),
+        ("spectral_coefficients", spectral_ascending, test_spectral_form_two_by_two_closed_form),
         ("sampled_fisher_norm_sq", sampled_missing_normalisation, test_sampled_estimator_hand_example),
         ("sampled_fisher_norm_sq", sampled_transposed_samples, lambda: test_sampled_estimator_equals_explicit_rank_one_sum(1)),
         ("sequence_gradients", seq_off_by_one, lambda: test_G_matches_four_loop_bruteforce_and_Kii_is_its_norm(0)),
