@@ -76,6 +76,7 @@ typedef enum {
 } isopo_variant;
 
 #define ISOPO_INFO_TIMEOUT 0x40000000
+#define ISOPO_INFO_NO_CONVERGENCE 0x20000000 /* isopo_transform_spectral: sweeps ran out; low bits = sweeps done */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 ISOPO_API const char* isopo_status_string(isopo_status s);
@@ -189,6 +190,34 @@ ISOPO_API isopo_status isopo_transform_advantages_batched(int n_layers, const fl
                                                           isopo_variant variant, const float* lambda,
                                                           const float* opt_pqr_regs, const float* const* states,
                                                           float* const* coeffs, int32_t* info, void* cuda_stream);
+
+/*
+ * isopo_transform_spectral: the interacting transform in the spectral form Alg. 2 prints,
+ *     K = U D U^T,   c = U ((1 / (D + lambda)) * (U^T A)),
+ * with the spectrum D as a second output (the quantity whose running mean regularises the
+ * interacting experiment of Sec. 4).  Eigen-directions with D_k <= rel_cutoff * max(D) are left out
+ * of the sum: rel_cutoff = 0 and a positive definite K give the coefficients of
+ * ISOPO_VAR_INTERACTING; lambda = 0 with a cut-off gives the pseudo-inverse on the kept range, which
+ * the Cholesky route cannot (it stops at a non-positive pivot).
+ *
+ * K is diagonalised by one-sided Jacobi rotations in float32 with float64 inner products, one CTA
+ * per call: milliseconds at B = 256, against ~0.1 ms for isopo_transform_advantages.  It is the
+ * diagnostic variant; its float32 eigenbasis limits the coefficients to a relative error of about
+ * 1e-7 * cond(K + lambda I) (kept range), the eigenvalues to ~1e-6 of the largest.
+ *
+ *   K            dev, float32 [B, B] row-major, symmetric (as written by isopo_layer_gram); B <= 256
+ *   A            dev, float32 [B]
+ *   lambda       >= 0;   rel_cutoff in [0, 1)
+ *   coeffs       dev, float32 [B], overwritten
+ *   eigenvalues  dev, float32 [B], from the largest down; may be NULL
+ *   ws           dev, isopo_spectral_workspace_bytes() bytes, 16-byte aligned; contents destroyed
+ * If the rotations have not died out after 30 sweeps, *info = ISOPO_INFO_NO_CONVERGENCE | sweeps
+ * and the outputs are those of the last sweep.
+ */
+ISOPO_API size_t isopo_spectral_workspace_bytes(void);
+ISOPO_API isopo_status isopo_transform_spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff,
+                                                float* coeffs, float* eigenvalues, void* ws, size_t ws_bytes,
+                                                int32_t* info, void* cuda_stream);
 
 /*
  * isopo_weight_grad: dW = beta * dW + sum_i coeffs[i] * G_i   (Alg. 1 "grad += advantages * rescaled

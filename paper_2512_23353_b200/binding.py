@@ -29,6 +29,7 @@ EXPORTS = (
     "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
     "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
     "isopo_reg_ema_update", "isopo_transform_advantages_rel", "isopo_transform_advantages_batched",
+    "isopo_spectral_workspace_bytes", "isopo_transform_spectral",
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
@@ -80,6 +81,11 @@ def _load():
     lib.isopo_transform_advantages_batched.restype = c.c_int
     lib.isopo_transform_advantages_batched.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_void_p,
                                                        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.isopo_spectral_workspace_bytes.restype = c.c_size_t
+    lib.isopo_spectral_workspace_bytes.argtypes = []
+    lib.isopo_transform_spectral.restype = c.c_int
+    lib.isopo_transform_spectral.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_float, c.c_float, c.c_void_p,
+                                             c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
     lib.isopo_transform_advantages_rel.restype = c.c_int
     lib.isopo_transform_advantages_rel.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
                                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -235,6 +241,26 @@ def isopo_transform_advantages_batched(Ks, A: torch.Tensor, variant: int, lams, 
                                                 s_ptrs.ctypes.data if s_ptrs is not None else None,
                                                 c_ptrs.ctypes.data, info.data_ptr(), _stream())
     _check(st, "isopo_transform_advantages_batched")
+
+
+INFO_NO_CONVERGENCE = 0x20000000
+
+
+def isopo_transform_spectral(K: torch.Tensor, A: torch.Tensor, lam: float, coeffs: torch.Tensor, info: torch.Tensor,
+                             rel_cutoff: float = 0.0, eigenvalues: torch.Tensor | None = None,
+                             ws: torch.Tensor | None = None) -> None:
+    """Interacting coefficients through the eigendecomposition of K (Alg. 2 as printed), optionally with the
+    spectrum (largest first) and with the directions below rel_cutoff * max(D) left out."""
+    B = A.numel()
+    assert K.dtype == torch.float32 and A.dtype == torch.float32 and coeffs.dtype == torch.float32
+    assert K.is_contiguous() and K.numel() == B * B and coeffs.numel() == B
+    assert eigenvalues is None or (eigenvalues.dtype == torch.float32 and eigenvalues.numel() == B)
+    if ws is None:
+        ws = torch.empty(lib.isopo_spectral_workspace_bytes(), dtype=torch.uint8, device=K.device)
+    st = lib.isopo_transform_spectral(K.data_ptr(), A.data_ptr(), B, float(lam), float(rel_cutoff), coeffs.data_ptr(),
+                                      eigenvalues.data_ptr() if eigenvalues is not None else None, ws.data_ptr(),
+                                      ws.numel(), info.data_ptr(), _stream())
+    _check(st, "isopo_transform_spectral")
 
 
 def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, seq_offsets, dW: torch.Tensor,

@@ -277,6 +277,19 @@ isopo_status isopo_transform_advantages_batched(int n_layers, const float* const
                            (cudaStream_t)cuda_stream);
 }
 
+size_t isopo_spectral_workspace_bytes(void) { return spectral_workspace_bytes(); }
+
+isopo_status isopo_transform_spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff,
+                                      float* coeffs, float* eigenvalues, void* ws, size_t ws_bytes, int32_t* info,
+                                      void* cuda_stream) {
+  if (!K || !A || !coeffs || !ws || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
+  if (!(lambda >= 0.0f) || !(rel_cutoff >= 0.0f && rel_cutoff < 1.0f)) return ISOPO_ERR_INVALID_ARG;
+  if ((uintptr_t)ws & 15) return ISOPO_ERR_INVALID_ARG;
+  if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  if (ws_bytes < spectral_workspace_bytes()) return ISOPO_ERR_WORKSPACE;
+  return spectral(K, A, B, lambda, rel_cutoff, coeffs, eigenvalues, ws, info, (cudaStream_t)cuda_stream);
+}
+
 isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
                                const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {

@@ -144,6 +144,9 @@ isopo_status transform(const float* K, const float* A, int B, isopo_variant v, f
 isopo_status transform_batched(int n, const float* const* K, const float* A, int B, isopo_variant v, const float* lambda,
                                const float* pqr_regs_host, const float* const* rel_state, float* const* coeffs,
                                int32_t* info, cudaStream_t st);
+size_t spectral_workspace_bytes();
+isopo_status spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff, float* coeffs, float* eig,
+                      void* ws, int32_t* info, cudaStream_t st);
 isopo_status reg_ema_update(const float* K, int B, float decay, float* state, cudaStream_t st);
 
 }  // namespace isopo
