@@ -49,7 +49,7 @@ extern "C" {
 typedef enum {
   ISOPO_OK = 0,
   ISOPO_ERR_INVALID_ARG = 1,  /* null pointer, bad size, bad offsets, misaligned buffer */
-  ISOPO_ERR_UNSUPPORTED = 2,  /* valid request that this build has no kernel for */
+  ISOPO_ERR_UNSUPPORTED = 2,  /* valid request that the library has no kernel for */
   ISOPO_ERR_WORKSPACE = 3,    /* ws_bytes smaller than isopo_workspace_bytes(...) */
   ISOPO_ERR_CUDA = 4          /* a CUDA runtime/driver call failed; see isopo_last_cuda_error() */
 } isopo_status;
