@@ -220,6 +220,22 @@ ISOPO_API isopo_status isopo_transform_spectral(const float* K, const float* A, 
                                                 int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_transform_spectral_batched: isopo_transform_spectral for several layers of one microbatch in
+ * one launch, one cluster per layer side by side (the decomposition is latency-bound, so n_layers
+ * of them take about the time of one).  Shared: A, B, rel_cutoff.
+ *
+ *   K, coeffs    HOST arrays of n_layers device pointers (1 <= n_layers <= ISOPO_MAX_BATCH)
+ *   lambda       HOST array of n_layers regularisers
+ *   eigenvalues  NULL, or HOST array of n_layers device pointers (entries may be NULL)
+ *   ws           dev, n_layers * isopo_spectral_workspace_bytes() bytes, 16-byte aligned
+ * A layer l that does not converge reports *info = ISOPO_INFO_NO_CONVERGENCE | (l << 16) | sweeps.
+ */
+ISOPO_API isopo_status isopo_transform_spectral_batched(int n_layers, const float* const* K, const float* A, int B,
+                                                        const float* lambda, float rel_cutoff, float* const* coeffs,
+                                                        float* const* eigenvalues, void* ws, size_t ws_bytes,
+                                                        int32_t* info, void* cuda_stream);
+
+/*
  * isopo_weight_grad: dW = beta * dW + sum_i coeffs[i] * G_i   (Alg. 1 "grad += advantages * rescaled
  * gradient" and "mod.grad += grad"; Alg. 2 "stack(seq_grads) @ advantages_preconditioned").
  *

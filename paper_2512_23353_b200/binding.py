@@ -29,7 +29,7 @@ EXPORTS = (
     "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
     "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
     "isopo_reg_ema_update", "isopo_transform_advantages_rel", "isopo_transform_advantages_batched",
-    "isopo_spectral_workspace_bytes", "isopo_transform_spectral",
+    "isopo_spectral_workspace_bytes", "isopo_transform_spectral", "isopo_transform_spectral_batched",
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
@@ -86,6 +86,10 @@ def _load():
     lib.isopo_transform_spectral.restype = c.c_int
     lib.isopo_transform_spectral.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_float, c.c_float, c.c_void_p,
                                              c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.isopo_transform_spectral_batched.restype = c.c_int
+    lib.isopo_transform_spectral_batched.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_void_p, c.c_float,
+                                                     c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
+                                                     c.c_void_p]
     lib.isopo_transform_advantages_rel.restype = c.c_int
     lib.isopo_transform_advantages_rel.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
                                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -261,6 +265,28 @@ def isopo_transform_spectral(K: torch.Tensor, A: torch.Tensor, lam: float, coeff
                                       eigenvalues.data_ptr() if eigenvalues is not None else None, ws.data_ptr(),
                                       ws.numel(), info.data_ptr(), _stream())
     _check(st, "isopo_transform_spectral")
+
+
+def isopo_transform_spectral_batched(Ks, A: torch.Tensor, lams, coeffs, info: torch.Tensor, rel_cutoff: float = 0.0,
+                                     eigenvalues=None, ws: torch.Tensor | None = None) -> None:
+    """isopo_transform_spectral for the layers Ks[l] -> coeffs[l] (and eigenvalues[l]) in one launch."""
+    n, B = len(Ks), A.numel()
+    assert len(coeffs) == n and len(lams) == n and (eigenvalues is None or len(eigenvalues) == n)
+    for K, co in zip(Ks, coeffs):
+        assert K.dtype == torch.float32 and K.is_contiguous() and K.numel() == B * B
+        assert co.dtype == torch.float32 and co.is_contiguous() and co.numel() == B
+    k_ptrs = np.array([K.data_ptr() for K in Ks], dtype=np.uint64)
+    c_ptrs = np.array([co.data_ptr() for co in coeffs], dtype=np.uint64)
+    e_ptrs = None
+    if eigenvalues is not None:
+        e_ptrs = np.array([e.data_ptr() if e is not None else 0 for e in eigenvalues], dtype=np.uint64)
+    lam = np.ascontiguousarray(np.asarray(lams, dtype=np.float32))
+    if ws is None:
+        ws = torch.empty(n * lib.isopo_spectral_workspace_bytes(), dtype=torch.uint8, device=A.device)
+    st = lib.isopo_transform_spectral_batched(n, k_ptrs.ctypes.data, A.data_ptr(), B, lam.ctypes.data, float(rel_cutoff),
+                                              c_ptrs.ctypes.data, e_ptrs.ctypes.data if e_ptrs is not None else None,
+                                              ws.data_ptr(), ws.numel(), info.data_ptr(), _stream())
+    _check(st, "isopo_transform_spectral_batched")
 
 
 def isopo_weight_grad(X: torch.Tensor, dY: torch.Tensor, coeffs: torch.Tensor, seq_offsets, dW: torch.Tensor,

@@ -290,6 +290,21 @@ isopo_status isopo_transform_spectral(const float* K, const float* A, int B, flo
   return spectral(K, A, B, lambda, rel_cutoff, coeffs, eigenvalues, ws, info, (cudaStream_t)cuda_stream);
 }
 
+isopo_status isopo_transform_spectral_batched(int n_layers, const float* const* K, const float* A, int B,
+                                              const float* lambda, float rel_cutoff, float* const* coeffs,
+                                              float* const* eigenvalues, void* ws, size_t ws_bytes, int32_t* info,
+                                              void* cuda_stream) {
+  if (n_layers < 1 || n_layers > ISOPO_MAX_BATCH) return ISOPO_ERR_INVALID_ARG;
+  if (!K || !A || !lambda || !coeffs || !ws || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
+  if (!(rel_cutoff >= 0.0f && rel_cutoff < 1.0f) || ((uintptr_t)ws & 15)) return ISOPO_ERR_INVALID_ARG;
+  if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  for (int l = 0; l < n_layers; ++l)
+    if (!K[l] || !coeffs[l] || !(lambda[l] >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
+  if (ws_bytes < (size_t)n_layers * spectral_workspace_bytes()) return ISOPO_ERR_WORKSPACE;
+  return spectral_batched(n_layers, K, A, B, lambda, rel_cutoff, coeffs, eigenvalues, ws, info,
+                          (cudaStream_t)cuda_stream);
+}
+
 isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
                                const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {

@@ -147,6 +147,9 @@ isopo_status transform_batched(int n, const float* const* K, const float* A, int
 size_t spectral_workspace_bytes();
 isopo_status spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff, float* coeffs, float* eig,
                       void* ws, int32_t* info, cudaStream_t st);
+isopo_status spectral_batched(int n, const float* const* K, const float* A, int B, const float* lambda,
+                              float rel_cutoff, float* const* coeffs, float* const* eig, void* ws, int32_t* info,
+                              cudaStream_t st);
 isopo_status reg_ema_update(const float* K, int B, float decay, float* state, cudaStream_t st);
 
 }  // namespace isopo

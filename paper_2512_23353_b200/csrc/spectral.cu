@@ -37,6 +37,17 @@ struct SpectralParams {
   float lambda, rel_cutoff;
 };
 
+// One launch serves up to ISOPO_MAX_BATCH layers that share A and B: cluster l works on layer l.
+struct SpectralBatch {
+  SpectralParams common;  // K, coeffs, eig, W, V, rotations, lambda are taken per layer
+  const float* K[ISOPO_MAX_BATCH];
+  float* coeffs[ISOPO_MAX_BATCH];
+  float* eig[ISOPO_MAX_BATCH];
+  float lambda[ISOPO_MAX_BATCH];
+  char* ws;          // layer l uses ws + l * ws_stride
+  size_t ws_stride;
+};
+
 __device__ __forceinline__ double warp_sum_d(double v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
@@ -77,11 +88,20 @@ __device__ __forceinline__ void cluster_barrier() {  // every thread of the clus
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-__global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kThreads) k_spectral(SpectralParams P) {
+__global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kThreads)
+k_spectral(const __grid_constant__ SpectralBatch batch) {
   __shared__ double s_d[kLd], s_f[kLd];
   __shared__ double s_fro2;
+  const int layer = blockIdx.x / kClusterSize, rank = blockIdx.x % kClusterSize;  // one cluster per layer
+  SpectralParams P = batch.common;
+  P.K = batch.K[layer];
+  P.coeffs = batch.coeffs[layer];
+  P.eig = batch.eig[layer];
+  P.lambda = batch.lambda[layer];
+  P.W = reinterpret_cast<float*>(batch.ws + (size_t)layer * batch.ws_stride);
+  P.V = P.W + (size_t)kLd * kLd;
+  P.rotations = reinterpret_cast<int*>(P.V + (size_t)kLd * kLd);
   const int B = P.B, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kThreads / 32;
-  const int rank = blockIdx.x;  // one cluster per launch
   const int gtid = rank * kThreads + tid, gthreads = kClusterSize * kThreads;
   float* W = P.W;  // read and written by every warp: no restrict, no read-only loads
   float* V = P.V;
@@ -149,7 +169,7 @@ __global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kThreads)
     ++sweeps;
   }
   if (rank != 0) return;  // the rest is one CTA's work
-  if (!converged && tid == 0) atomicCAS(P.info, 0, ISOPO_INFO_NO_CONVERGENCE | sweeps);
+  if (!converged && tid == 0) atomicCAS(P.info, 0, ISOPO_INFO_NO_CONVERGENCE | (layer << 16) | sweeps);
 
   // d_k = v_k . w_k (= v_k^T K v_k), y_k = v_k . A
   for (int k = warp; k < B; k += nwarps) {
@@ -189,19 +209,33 @@ __global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kThreads)
 
 size_t spectral_workspace_bytes() { return sizeof(float) * 2 * (size_t)kLd * kLd + 256; }
 
-isopo_status spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff, float* coeffs, float* eig,
-                      void* ws, int32_t* info, cudaStream_t st) {
+isopo_status spectral_batched(int n, const float* const* K, const float* A, int B, const float* lambda,
+                              float rel_cutoff, float* const* coeffs, float* const* eig, void* ws, int32_t* info,
+                              cudaStream_t st) {
   if (B > kLd) return ISOPO_ERR_UNSUPPORTED;
-  float* W = (float*)ws;
-  int* rotations = (int*)(W + 2 * (size_t)kLd * kLd);
-  ISOPO_CUDA_TRY(cudaMemsetAsync(rotations, 0, sizeof(int), st));
-  SpectralParams P{K, A, coeffs, eig, W, W + (size_t)kLd * kLd, rotations, info, B, lambda, rel_cutoff};
+  SpectralBatch T{};
+  T.common.A = A; T.common.info = info; T.common.B = B; T.common.rel_cutoff = rel_cutoff;
+  T.ws = (char*)ws;
+  T.ws_stride = spectral_workspace_bytes();
+  for (int l = 0; l < n; ++l) {
+    T.K[l] = K[l];
+    T.coeffs[l] = coeffs[l];
+    T.eig[l] = eig ? eig[l] : nullptr;
+    T.lambda[l] = lambda[l];
+    // the rotation counter of layer l sits behind its W and V
+    ISOPO_CUDA_TRY(cudaMemsetAsync(T.ws + (size_t)l * T.ws_stride + sizeof(float) * 2 * (size_t)kLd * kLd, 0, sizeof(int), st));
+  }
   {
     LaunchScope scope(kIdTransform, st);
-    k_spectral<<<kClusterSize, kThreads, 0, st>>>(P);
+    k_spectral<<<n * kClusterSize, kThreads, 0, st>>>(T);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
+}
+
+isopo_status spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff, float* coeffs, float* eig,
+                      void* ws, int32_t* info, cudaStream_t st) {
+  return spectral_batched(1, &K, A, B, &lambda, rel_cutoff, &coeffs, eig ? &eig : nullptr, ws, info, st);
 }
 
 }  // namespace isopo

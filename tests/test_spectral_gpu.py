@@ -103,3 +103,34 @@ def test_time_at_full_size_and_argument_checks(b, capsys):
     big = torch.eye(300, device="cuda")
     with pytest.raises(b.IsopoError):
         b.isopo_transform_spectral(big, torch.ones(300, device="cuda"), lam, torch.empty(300, device="cuda"), info)
+
+
+def test_seven_layers_in_one_launch(b, capsys):
+    """The block's seven K in one launch, one cluster per layer: the same results as seven calls, in
+    about the time of one."""
+    B, n = 256, 7
+    Ks = [torch.from_numpy(_gram(B, 1 + l % 3, 900 + l) * np.float32(1 + l)).cuda() for l in range(n)]
+    A = torch.from_numpy(np.random.default_rng(5).standard_normal(B).astype(np.float32)).cuda()
+    lams = [float(1e-3 * torch.diagonal(K).mean().item()) for K in Ks]
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cs = [torch.empty(B, device="cuda") for _ in range(n)]
+    es = [torch.empty(B, device="cuda") if l % 2 == 0 else None for l in range(n)]
+    b.isopo_transform_spectral_batched(Ks, A, lams, cs, info, eigenvalues=es)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    b.isopo_transform_spectral_batched(Ks, A, lams, cs, info, eigenvalues=es)
+    torch.cuda.synchronize()
+    ms = (time.perf_counter() - t0) * 1e3
+    with capsys.disabled():
+        print(f"\n[isopo_transform_spectral_batched, 7 x B = 256: {ms:.2f} ms]")
+    assert int(info.item()) == 0
+    for l in range(n):
+        c1, e1 = torch.empty(B, device="cuda"), torch.empty(B, device="cuda")
+        b.isopo_transform_spectral(Ks[l], A, lams[l], c1, info, eigenvalues=e1)
+        torch.cuda.synchronize()
+        assert torch.equal(c1, cs[l])
+        if es[l] is not None:
+            assert torch.equal(e1, es[l])
+    assert int(info.item()) == 0
+    with pytest.raises(b.IsopoError):
+        b.isopo_transform_spectral_batched(Ks, A, lams, cs, info, ws=torch.empty(1024, dtype=torch.uint8, device="cuda"))
