@@ -123,6 +123,28 @@ ISOPO_API isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dty
                               size_t ws_bytes, int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_layer_gram_shared_x: isopo_layer_gram on the Gram route for up to three projections that
+ * read the SAME input X (q/k/v, gate/up of a transformer block): K^(h) = layer NTK of projection h
+ * (Eq. one / Eq. two per layer).  The token Gram X X^T is formed once per pair of token tiles and
+ * multiplied with each projection's dY^(h) dY^(h)^T, so the X contraction and the loads of X are paid
+ * once instead of n_proj times.  bfloat16 only; results as n_proj calls of isopo_layer_gram with
+ * ISOPO_PATH_GRAM (float atomics: not bit-identical).
+ *
+ *   X        dev, bf16 [T, d_in]
+ *   n_proj   1 .. 3
+ *   dY       HOST array of n_proj device pointers, dY[h] bf16 [T, d_out[h]]
+ *   d_out    HOST array of n_proj widths (multiples of 8)
+ *   K        HOST array of n_proj device pointers, each float32 [B, B], overwritten
+ *   ws       dev, isopo_workspace_bytes(dtype, T, d_in, max_h d_out[h], B, ISOPO_PATH_GRAM) bytes, 1024-byte aligned
+ * Follow it with isopo_weight_grad(X, dY[h], ..., ISOPO_PATH_GRAM, ...) per projection (each with a
+ * workspace of its own size; the call refreshes what it needs).
+ */
+ISOPO_API isopo_status isopo_layer_gram_shared_x(const void* X, int n_proj, const void* const* dY, const int* d_out,
+                                                 isopo_dtype dtype, int64_t T, int d_in,
+                                                 const int64_t* seq_offsets_host, int B, float* const* K, void* ws,
+                                                 size_t ws_bytes, int32_t* info, void* cuda_stream);
+
+/*
  * isopo_transform_advantages: advantages A -> coefficients c (dW = sum_i c_i G_i).
  *
  * With F_i^2 = sum_j K_ij^2 / sum_j K_jj (the Fisher norm of Eq. F-norm-basic evaluated with the B

@@ -207,6 +207,28 @@ isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, 
   return bf16_ntk(G, L, B, K, info, st);
 }
 
+isopo_status isopo_layer_gram_shared_x(const void* X, int n_proj, const void* const* dY, const int* d_out, isopo_dtype dtype,
+                                       int64_t T, int d_in, const int64_t* seq_offsets_host, int B, float* const* K,
+                                       void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  if (!dY || !d_out || !K || !info || n_proj < 1 || n_proj > 3) return ISOPO_ERR_INVALID_ARG;
+  if (dtype != ISOPO_BF16) return ISOPO_ERR_UNSUPPORTED;
+  int d_max = 0;
+  for (int h = 0; h < n_proj; ++h) {
+    if (!K[h]) return ISOPO_ERR_INVALID_ARG;
+    isopo_status s = check_layer_args(X, dY[h], dtype, T, d_in, d_out[h], seq_offsets_host, B, ISOPO_PATH_GRAM, ws);
+    if (s != ISOPO_OK) return s;
+    d_max = std::max(d_max, d_out[h]);
+  }
+  const WsLayout L = ws_layout(dtype, T, d_in, d_max, B, ISOPO_PATH_GRAM);
+  if (ws_bytes < L.total) return ISOPO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* w = (char*)ws;
+  int32_t* tokseq = (int32_t*)(w + L.off_tokseq);
+  isopo_status s = launch_prep(seq_offsets_host, B, T, (int64_t*)(w + L.off_offsets), tokseq, st);
+  if (s != ISOPO_OK) return s;
+  return bf16_gram_shared(X, dY, T, d_in, d_out, n_proj, tokseq, B, K, info, st);
+}
+
 size_t isopo_sampled_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, int n_samples) {
   if (!sizes_ok(dtype, T, d_in, d_out, B) || n_samples < 1 || n_samples > ISOPO_MAX_SAMPLES) return 0;
   return sampled_layout(dtype, T, d_in, d_out, B, n_samples).total;

@@ -124,6 +124,8 @@ isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out,
                           float beta, cudaStream_t st);
 isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
                        float* K, int32_t* info, cudaStream_t st);
+isopo_status bf16_gram_shared(const void* X, const void* const* dY, int64_t T, int d_in, const int* d_out, int n_heads,
+                              const int32_t* tokseq, int B, float* const* K, int32_t* info, cudaStream_t st);
 isopo_status bf16_weight_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const float* tokscale,
                               void* scaled, float* dW, float beta, int32_t* info, cudaStream_t st);
 

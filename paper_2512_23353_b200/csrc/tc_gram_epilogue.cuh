@@ -45,12 +45,14 @@ __device__ __forceinline__ void decode_pair_strips(long long u, int nT, int S, i
 // Strip width for tiles of `tile_bytes` (both operands' rows of one tile): column and row tiles of
 // ~148 concurrent units should stay within about 48 MB.
 inline int gram_strip_width(double tile_bytes, int concurrent_units) {
-  int best = 2;
+  int best = 0, fewest = 2;
+  double fewest_tiles = 1e300;
   for (int S = 2; S <= 32; ++S) {
     const double tiles = S + (double)concurrent_units / S;
     if (tiles * tile_bytes <= 48e6) best = S;  // widest strip that still fits (fewer, longer strips)
+    if (tiles < fewest_tiles) { fewest_tiles = tiles; fewest = S; }
   }
-  return best;
+  return best ? best : fewest;  // nothing fits: the strip with the fewest tiles in flight
 }
 
 struct RowSegments {
