@@ -175,6 +175,43 @@ def oracle_sample(workload_name: str, n_seq: int, len_div: int):
     return T, dt, desc
 
 
+def parity_check(layers, off, A, lam_by_layer, variant_name, n_seq=8):
+    """The last timed step's outputs against the fp64 oracle, the cheap way: per projection, K_ij for all
+    pairs of the `n_seq` shortest sequences (their G_i materialised in float64), one 32 x 64 block of dW over
+    ALL sequences with the library's coefficients, and those coefficients against the oracle's transform of
+    the library's K.  Relative Frobenius errors, the worst projection of each; tolerance 2e-2 (bf16) / 1e-5."""
+    import torch
+
+    from oracle import isopo_oracle as orc
+
+    def f64(t):
+        return t.detach().to("cpu").to(torch.float64).numpy()
+
+    def rel(a, ref):
+        return float(np.linalg.norm(np.asarray(a, np.float64) - ref) / max(np.linalg.norm(ref), 1e-300))
+
+    L_len = np.diff(off)
+    pick = sorted(np.argsort(L_len, kind="stable")[:n_seq].tolist())
+    off_s = np.concatenate([[0], np.cumsum([L_len[i] for i in pick])]).astype(np.int64)
+    rng = np.random.default_rng(11)
+    worst = {"K": 0.0, "dW": 0.0, "c_from_K": 0.0}
+    t0 = time.perf_counter()
+    for L, lam in zip(layers, lam_by_layer):
+        lay = L["layer"]
+        rows = torch.cat([torch.arange(int(off[i]), int(off[i + 1])) for i in pick]).to(L["X"].device)
+        G_s = orc.sequence_gradients(f64(L["X"][rows]), f64(L["dY"][rows]), off_s)
+        worst["K"] = max(worst["K"], rel(f64(L["K"])[np.ix_(pick, pick)], orc.ntk(G_s)))
+        del G_s
+        m_idx = torch.from_numpy(np.sort(rng.choice(lay.d_out, size=min(32, lay.d_out), replace=False))).to(L["X"].device)
+        n_idx = torch.from_numpy(np.sort(rng.choice(lay.d_in, size=min(64, lay.d_in), replace=False))).to(L["X"].device)
+        G_blk = orc.sequence_gradients(f64(L["X"][:, n_idx]), f64(L["dY"][:, m_idx]), off)
+        worst["dW"] = max(worst["dW"], rel(f64(L["dW"][m_idx][:, n_idx]), orc.weight_gradient(G_blk, f64(L["c"]))))
+        worst["c_from_K"] = max(worst["c_from_K"],
+                                rel(f64(L["c"]), orc.transform_advantages(f64(L["K"]), f64(A), variant_name, lam)))
+    return {**worst, "sequences_in_K_sample": len(pick), "dW_block": "32 x 64 over all sequences",
+            "projections": len(layers), "seconds": time.perf_counter() - t0}
+
+
 def cpu_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -350,6 +387,16 @@ def run_gpu(args):
     elapsed_ms, total_tokens = reduce_over_ranks(elapsed_ms, float(T), dev)
     ms_per_step = elapsed_ms / args.steps
     value = total_tokens / (ms_per_step / 1000.0)
+
+    # ---- the timed run's own outputs against the oracle (rank 0; stored route: K, c, dW are all there) ----
+    parity = None
+    if rank == 0 and not sampled and not args.skip_parity:
+        from oracle import isopo_oracle as orc
+        parity = parity_check(layers, off, A, [L["lam"] for L in layers],
+                              orc.INTERACTING if args.variant == "interacting" else orc.NORMALISED)
+        tol = 2e-2 if w.dtype == "bf16" else 1e-5
+        parity["tolerance"] = tol
+        parity["ok"] = bool(parity["K"] <= tol and parity["dW"] <= tol and parity["c_from_K"] <= max(tol * 1e-2, 1e-5))
 
     if rank != 0:
         if world > 1:
@@ -545,12 +592,77 @@ def run_gpu(args):
                "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": n_e2e}
         del pinned, dW_host
 
+    # ---- the other route through the library on the same inputs: Algorithm 1 as printed (sampled Fisher norm) ----
+    routes = None
+    if not sampled and w.dtype == "bf16" and world == 1 and not args.skip_routes:
+        s_ws = aligned(max(b.isopo_sampled_workspace_bytes(dt_code, T, L["layer"].d_in, L["layer"].d_out, B, len(sample_rows))
+                           for L in layers))
+        F2 = torch.zeros(B, dtype=torch.float32, device=dev)
+        lam_s = {}
+
+        def sampled_step():
+            for L in layers:
+                b.isopo_sampled_coefficients(L["X"], L["dY"], off, sample_rows, A, lam_s.get(id(L), 0.0), L["c"], s_ws, info, F2)
+                b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], s_ws, info, b.PATH_GRAM, 0.0)
+
+        for L in layers:  # regulariser 1e-3 * mean(F^2), taken once from an untimed pass
+            b.isopo_sampled_coefficients(L["X"], L["dY"], off, sample_rows, A, 0.0, L["c"], s_ws, info, F2)
+            lam_s[id(L)] = 1e-3 * float(F2.mean().item())
+        for _ in range(3):
+            sampled_step()
+        torch.cuda.synchronize()
+        b.isopo_profile_collect()
+        n_s = max(1, min(args.steps, 10))
+        s_sampler = ClockSampler(local)
+        b.isopo_profile_enable(True)
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        s_sampler.start()
+        a.record()
+        for _ in range(n_s):
+            sampled_step()
+        c.record()
+        torch.cuda.synchronize()
+        s_clocks = s_sampler.stop()
+        b.isopo_profile_enable(False)
+        s_prof = b.isopo_profile_collect()
+        if int(info.item()) != 0:
+            raise SystemExit(f"device-side error on the sampled route: info={int(info.item()):#x}")
+        s_ms = a.elapsed_time(c) / n_s
+        routes = {"sampled": {
+            "what": "Algorithm 1 as printed: isopo_sampled_coefficients (%d seeded token samples) + isopo_weight_grad on "
+                    "the GEMM route for each projection; normalised variant; same inputs, same run" % len(sample_rows),
+            "ms_per_step": s_ms, "steps": n_s, "tokens_per_s": T / (s_ms * 1e-3),
+            "overhead_vs_plain_dw_gemm": s_ms / plain_ms,
+            "kernels": {k: {"ms_per_step": v[0] / n_s, "launches_per_step": v[1] / n_s} for k, v in s_prof.items()},
+            "clocks": s_clocks}}
+        del s_ws
+
     # ---- the oracle on this machine's host cores, bounded sample ----
     cpu = None
     if world == 1 and not args.skip_cpu:
         tok_s, dt_s, desc = oracle_sample(args.workload, args.cpu_seqs, args.cpu_len_div)
         cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
                "seconds": dt_s}
+
+    # ---- end-to-end decoder backward (library calls in every linear layer's hook) against plain gradients ----
+    cfg_layers = [f"{L['layer'].name}:{L['layer'].d_in}->{L['layer'].d_out}" for L in layers]
+    cfg_paths = ["gram" if L["path"] == b.PATH_GRAM else "materialise" for L in layers]
+    decoder = None
+    if world == 1 and not args.skip_decoder and args.workload == "llm_1p5b" and not args.layers and not args.seqs:
+        import bench_decoder
+        for L in layers:  # the block's tensors and workspaces go first: the decoder needs the memory
+            L.clear()
+        del layers
+        torch.cuda.empty_cache()
+        decoder = {}
+        for route in ("stored", "sampled"):
+            d_sampler = ClockSampler(local)
+            d_sampler.start()
+            rec = bench_decoder.run_decoder(bench_decoder.parse_args(["--route", route, "--steps", "2", "--warmup", "1"]), dev)
+            rec["clocks"] = d_sampler.stop()
+            decoder[route] = rec
+            torch.cuda.empty_cache()
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -559,8 +671,7 @@ def run_gpu(args):
         "config": {"workload": args.workload, "B": B, "tokens": T,
                    "route": "sampled (Algorithm 1, %d token samples)" % len(sample_rows) if sampled else "stored gradients",
                    "variant": "normalised (Algorithm 1)" if sampled else args.variant,
-                   "layers": [f"{L['layer'].name}:{L['layer'].d_in}->{L['layer'].d_out}" for L in layers],
-                   "paths": ["gram" if L["path"] == b.PATH_GRAM else "materialise" for L in layers],
+                   "layers": cfg_layers, "paths": cfg_paths,
                    "l2": ("L2 flushed between steps (256 MB fill, untimed); every step timed by its own events"
                           if flush else "inputs larger than L2 (no flush needed)"),
                    "step": ("sampled_coefficients + weight_grad for each projection" if sampled else
@@ -574,6 +685,9 @@ def run_gpu(args):
         "gpu_launches": int(sum(v[1] for v in prof.values())),
         "roofline": roofline,
         "cpu_baseline": cpu,
+        "parity": parity,
+        "routes": routes,
+        "decoder": decoder,
         "step_tflops": step_tflops,
         "pct_bf16_peak_sustained": step_tflops / peaks["bf16_tflops_sustained"],
         "plain_dw_gemm_ms": plain_ms,
@@ -606,6 +720,9 @@ def main():
                     help="also capture one step in a CUDA graph and time its replays (reported under cuda_graph)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-parity", action="store_true", help="do not check the timed run's outputs against the oracle")
+    ap.add_argument("--skip-routes", action="store_true", help="do not also time the sampled route (Algorithm 1)")
+    ap.add_argument("--skip-decoder", action="store_true", help="do not run the end-to-end decoder harness")
     ap.add_argument("--layers", default="", help="comma-separated projection names (default: all of the block)")
     ap.add_argument("--seqs", type=int, default=0, help="use only the first N sequences (profiling aid)")
     ap.add_argument("--short-warmup", action="store_true", help="allow fewer than 3 warm-up steps (profiling only)")

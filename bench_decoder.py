@@ -189,7 +189,7 @@ def group_advantages(B, group, rng):
     return A.reshape(-1)[:B].astype(np.float32)
 
 
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--layers", type=int, default=24)
     ap.add_argument("--d-model", type=int, default=2048)
@@ -204,9 +204,12 @@ def main():
     ap.add_argument("--samples", type=int, default=128)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
-    args = ap.parse_args()
+    return ap.parse_args(argv)
 
-    dev = torch.device("cuda", 0)
+
+def run_decoder(args, dev=None):
+    """Both arms on one device; returns the record that main() prints."""
+    dev = dev or torch.device("cuda", torch.cuda.current_device())
     torch.cuda.set_device(dev)
     rng = np.random.default_rng(1005)
     lengths = rng.integers(args.len_lo, args.len_hi + 1, size=args.seqs)
@@ -254,7 +257,11 @@ def main():
         "tokens_per_s_isopo": mb.T / ((ours["fwd"] + ours["bwd"]) * 1e-3),
         "peak_mem_gb": torch.cuda.max_memory_allocated() / 2 ** 30,
     }
-    print(json.dumps(out))
+    return out
+
+
+def main():
+    print(json.dumps(run_decoder(parse_args())))
 
 
 if __name__ == "__main__":

@@ -28,7 +28,19 @@
  *     not positive definite (interacting transform); ISOPO_INFO_TIMEOUT | id = a bounded wait inside
  *     kernel `id` ran out.  The library only ever overwrites a zero `*info`.  When `*info` != 0 the
  *     outputs are unspecified (but every access stayed in bounds).
- *   - There is no CPU fallback and no global state; one GPU.
+ *   - There is no CPU fallback; one GPU per call (the current device).
+ *   - Process-wide state, all of it host side: the measurement hooks' event list (isopo_profile_*), the
+ *     deterministic-mode switch (isopo_set_deterministic), per-device caches of launch limits, and the
+ *     device address of isopo_layer_gram_static's scratch.  Host threads: isopo_status_string,
+ *     isopo_kernel_name, isopo_choose_path, the *_workspace_bytes queries and isopo_last_cuda_error
+ *     (thread-local) may be called from any thread at any time.  The entry points that enqueue work may
+ *     be called from several host threads at once as long as profiling is disabled, no thread changes
+ *     the deterministic-mode switch meanwhile, and each thread uses its own workspace, outputs and
+ *     `info`; the per-device caches are filled with identical values by whichever thread comes first.
+ *     isopo_profile_enable / isopo_profile_collect, isopo_set_deterministic and
+ *     isopo_layer_gram_static (it pauses profiling and shares one scratch array) must not run
+ *     concurrently with any other call of the library.
+ *   - Under a profiler every entry point that enqueues work shows as an NVTX range of its own name.
  */
 #ifndef ISOPO_H_
 #define ISOPO_H_
@@ -77,6 +89,8 @@ typedef enum {
 
 #define ISOPO_INFO_TIMEOUT 0x40000000
 #define ISOPO_INFO_NO_CONVERGENCE 0x20000000 /* isopo_transform_spectral: sweeps ran out; low bits = sweeps done */
+#define ISOPO_INFO_BOUNDS 0x08000000 /* debug build only (isopo_debug_build): kernel `id` computed an index outside its buffer; the access was skipped */
+#define ISOPO_INFO_STALE_WORKSPACE 0x10000000 /* isopo_weight_grad(MATERIALISE): the workspace holds another layer's or microbatch's gradients */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 ISOPO_API const char* isopo_status_string(isopo_status s);
@@ -222,8 +236,8 @@ ISOPO_API isopo_status isopo_transform_advantages_batched(int n_layers, const fl
  * ISOPO_VAR_INTERACTING; lambda = 0 with a cut-off gives the pseudo-inverse on the kept range, which
  * the Cholesky route cannot (it stops at a non-positive pivot).
  *
- * K is diagonalised by one-sided Jacobi rotations in float32 with float64 inner products, one CTA
- * per call: milliseconds at B = 256, against ~0.1 ms for isopo_transform_advantages.  It is the
+ * K is diagonalised by one-sided Jacobi rotations in float32 with float64 inner products, a cluster
+ * of eight CTAs per K: milliseconds at B = 256, against ~0.1 ms for isopo_transform_advantages.  It is the
  * diagnostic variant; its float32 eigenbasis limits the coefficients to a relative error of about
  * 1e-7 * cond(K + lambda I) (kept range), the eigenvalues to ~1e-6 of the largest.
  *
@@ -262,10 +276,15 @@ ISOPO_API isopo_status isopo_transform_spectral_batched(int n_layers, const floa
  * gradient" and "mod.grad += grad"; Alg. 2 "stack(seq_grads) @ advantages_preconditioned").
  *
  * `path` must be the value given to isopo_layer_gram for this layer (AUTO resolves identically).
- * MATERIALISE: streams the G_i left in the workspace by isopo_layer_gram.  GRAM: one GEMM over all
- * tokens, dW = (coeffs[seq(t)] * dY)^T X, with the per-token scale applied to the narrower operand
- * (rounded to nearest even in bf16) in one pass before the GEMM, or, for small layers, to the rows
- * as they land in shared memory.
+ * MATERIALISE: streams the G_i left in the workspace by isopo_layer_gram.  The workspace carries a
+ * tag (dtype, T, d_in, d_out, B, a hash of the offsets) written by that call; if this call's
+ * arguments do not match it, dW is left untouched and *info = ISOPO_INFO_STALE_WORKSPACE.
+ * GRAM: one GEMM over all tokens, dW = (coeffs[seq(t)] * dY)^T X.  bf16, layers whose wider side is
+ * at most 2048 (and sequences of about 100 tokens or more): every run of tokens of one sequence is
+ * accumulated on its own in tensor memory and multiplied by its coefficient when the accumulator
+ * is drained, so no operand is rounded a second time.  Wider bf16 layers: the per-token scale is
+ * applied to the narrower operand (rounded to nearest even in bf16) in one pass before a plain
+ * GEMM, or, for layers with few rows, to the rows as they land in shared memory.
  *
  *   coeffs  dev, float32 [B]
  *   dW      dev, float32 [d_out, d_in] row-major (the layout of `grad_out.T @ act_in`)
@@ -329,7 +348,9 @@ ISOPO_API isopo_status isopo_sampled_coefficients(const void* X, const void* dY,
  * The first call on each device looks up the array's device address (one cudaGetSymbolAddress with
  * that device current); make that first call outside any stream capture.  All calls on a device
  * share the one array: calls whose kernels could overlap on the GPU (different streams, no
- * ordering between them) race on it and must be serialised by the caller.  The array keeps what
+ * ordering between them) race on it and must be serialised by the caller.  On the host the call is
+ * not thread-safe against any other call of the library either (it pauses the process-wide event
+ * timing for its duration and fills the address cache unlocked).  The array keeps what
  * the previous call left; every part that is read is rewritten or cleared first.
  *
  * Arguments and the result are those of isopo_layer_gram with path = ISOPO_PATH_GRAM; K agrees
@@ -342,13 +363,46 @@ ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, is
                                                int32_t* info, void* cuda_stream);
 
 /*
+ * Deterministic mode (the paper has no counterpart; a diagnostic that tells a race from rounding).
+ * Normally K of the bf16 MATERIALISE route is summed over the CTAs with float atomics, so two runs
+ * differ in the last bits.  With the mode on, every CTA stores its partial K in the workspace and a
+ * second kernel adds the partials in a fixed order: K, the coefficients and dW of that route are
+ * then bit-identical from run to run.  The switch is process-wide and changes
+ * isopo_workspace_bytes(..., MATERIALISE) (160 * B * B * 4 more bytes for bf16): set it before
+ * sizing workspaces.  The GRAM route and the GEMM-route weight gradient keep their float atomics.
+ *
+ * isopo_debug_build() is 1 when the library was compiled with -DISOPO_DEBUG (libisopo_debug.so): every
+ * data-dependent index of the kernels is then range-checked before use, a violation skips the access
+ * and sets *info = ISOPO_INFO_BOUNDS | kernel id.
+ */
+ISOPO_API void isopo_set_deterministic(int on);
+ISOPO_API int isopo_get_deterministic(void);
+ISOPO_API int isopo_debug_build(void);
+
+/*
+ * isopo_selftest_bounded_wait (the paper has no counterpart): runs the library's bounded mbarrier wait
+ * on a barrier that nothing ever arrives on, in a kernel that owns no TMA copy and no tensor memory,
+ * so that the give-up path of the tensor-core kernels can be exercised without hanging or faulting
+ * anything.  After synchronising the stream: *info == (ISOPO_INFO_TIMEOUT | kernel id of
+ * "k_wait_probe"), *roles_at_teardown == 3 (the role that timed out, the role that saw its abort
+ * flag, and the role without waits all reached the common teardown), and the context is as usable as
+ * before.
+ *
+ *   limit_clocks       1 .. 2^28 SM clock ticks the first role waits before it gives up (1e5 = ~50 us)
+ *   info               dev int32, zeroed by the caller
+ *   roles_at_teardown  dev int32, overwritten
+ */
+ISOPO_API isopo_status isopo_selftest_bounded_wait(int64_t limit_clocks, int32_t* info, int32_t* roles_at_teardown,
+                                                   void* cuda_stream);
+
+/*
  * Measurement hooks (the paper has no counterpart).  While enabled, every kernel the library
  * launches is bracketed by CUDA events on its stream.  isopo_profile_collect synchronises those
  * events, adds the elapsed milliseconds and launch counts per kernel into the caller's arrays
  * (host, ISOPO_NUM_KERNELS entries each, overwritten) and forgets them.  Launch counts are kept
  * even while event timing is disabled.  Not thread-safe; meant for benchmarks.
  */
-#define ISOPO_NUM_KERNELS 16
+#define ISOPO_NUM_KERNELS 17
 ISOPO_API void isopo_profile_enable(int on);
 ISOPO_API isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_kernel);
 ISOPO_API const char* isopo_kernel_name(int kernel_id);

@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libisopo.so")
+# ISOPO_LIB_VARIANT=debug selects the range-checking build (libisopo_debug.so, `build(debug=True)`)
+LIB_PATH = os.path.join(_PKG, "libisopo_debug.so" if os.environ.get("ISOPO_LIB_VARIANT") == "debug" else "libisopo.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
 F32, BF16 = 0, 1
@@ -22,6 +23,7 @@ PATH_AUTO, PATH_GRAM, PATH_MATERIALISE = 0, 1, 2
 (VAR_REINFORCE, VAR_NORMALISED, VAR_DIRECTION, VAR_EUCLID, VAR_GENERAL, VAR_INTERACTING,
  VAR_NORMALISED_RAW) = range(7)
 INFO_TIMEOUT = 0x40000000
+INFO_STALE_WORKSPACE = 0x10000000
 
 EXPORTS = (
     "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",
@@ -30,10 +32,11 @@ EXPORTS = (
     "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
     "isopo_reg_ema_update", "isopo_transform_advantages_rel", "isopo_transform_advantages_batched",
     "isopo_spectral_workspace_bytes", "isopo_transform_spectral", "isopo_transform_spectral_batched",
+    "isopo_selftest_bounded_wait", "isopo_set_deterministic", "isopo_get_deterministic", "isopo_debug_build",
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
-NUM_KERNELS = 16
+NUM_KERNELS = 17
 
 
 class IsopoError(RuntimeError):
@@ -97,6 +100,14 @@ def _load():
     lib.isopo_transform_advantages_rel.restype = c.c_int
     lib.isopo_transform_advantages_rel.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
                                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.isopo_set_deterministic.restype = None
+    lib.isopo_set_deterministic.argtypes = [c.c_int]
+    lib.isopo_get_deterministic.restype = c.c_int
+    lib.isopo_get_deterministic.argtypes = []
+    lib.isopo_debug_build.restype = c.c_int
+    lib.isopo_debug_build.argtypes = []
+    lib.isopo_selftest_bounded_wait.restype = c.c_int
+    lib.isopo_selftest_bounded_wait.argtypes = [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.isopo_profile_enable.restype = None
     lib.isopo_profile_enable.argtypes = [c.c_int]
     lib.isopo_profile_collect.restype = c.c_int
@@ -350,6 +361,21 @@ def isopo_sampled_coefficients(X: torch.Tensor, dY: torch.Tensor, seq_offsets, s
                                         coeffs.data_ptr(), F2.data_ptr() if F2 is not None else None, ws.data_ptr(),
                                         ws.numel(), info.data_ptr(), _stream())
     _check(st, "isopo_sampled_coefficients")
+
+
+def isopo_set_deterministic(on: bool) -> None:
+    lib.isopo_set_deterministic(1 if on else 0)
+
+
+def isopo_debug_build() -> bool:
+    return bool(lib.isopo_debug_build())
+
+
+def isopo_selftest_bounded_wait(limit_clocks: int, info: torch.Tensor, roles_at_teardown: torch.Tensor) -> None:
+    """Makes one bounded mbarrier wait run out (nothing ever arrives) and lets the kernel tear down."""
+    assert info.dtype == torch.int32 and roles_at_teardown.dtype == torch.int32
+    _check(lib.isopo_selftest_bounded_wait(int(limit_clocks), info.data_ptr(), roles_at_teardown.data_ptr(), _stream()),
+           "isopo_selftest_bounded_wait")
 
 
 def isopo_profile_enable(on: bool) -> None:

@@ -6,9 +6,18 @@
 #include <algorithm>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "isopo_internal.h"
 
 namespace isopo {
+
+// NVTX range named after the entry point, open for the duration of the host call (the kernels it
+// enqueues appear under it in a profiler's timeline; without a profiler attached this is a no-op).
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+};
 
 static thread_local char g_cuda_err[256] = "no error";
 
@@ -18,6 +27,9 @@ void set_cuda_error(cudaError_t e, const char* where) {
   else
     snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
 }
+
+static bool g_deterministic = false;
+bool deterministic_mode() { return g_deterministic; }
 
 // ---- measurement hooks ----
 struct ProfRecord { int id; cudaEvent_t a, b; };
@@ -57,6 +69,8 @@ ProfilingPause::~ProfilingPause() { g_prof_on = was_on_; }
 WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path resolved) {
   WsLayout L{};
   size_t p = 0;
+  L.off_tag = p;
+  p = align_up(p + sizeof(WsTag), 1024);
   L.off_offsets = p;
   p = align_up(p + sizeof(int64_t) * (size_t)(B + 1), 1024);
   L.off_order = p;
@@ -74,13 +88,29 @@ WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, iso
     L.tiles_n = (d_in + kTileN - 1) / kTileN;
     L.n_pad = (int64_t)L.tiles_m * L.tiles_n * kTileElems;
     if (resolved == ISOPO_PATH_MATERIALISE) p = align_up(p + (size_t)2 * (size_t)B * (size_t)L.n_pad, 1024);
+    L.off_kpart = p;
+    if (resolved == ISOPO_PATH_MATERIALISE && deterministic_mode())
+      p = align_up(p + sizeof(float) * (size_t)kNtkMaxPartials * (size_t)B * (size_t)B, 1024);
   } else {
     L.tiles_m = L.tiles_n = 0;
+    L.off_kpart = p;
     L.n_pad = (int64_t)d_in * d_out;
     if (resolved == ISOPO_PATH_MATERIALISE) p = align_up(p + (size_t)4 * (size_t)B * (size_t)L.n_pad, 1024);
   }
   L.total = p;
   return L;
+}
+
+WsTag make_ws_tag(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, const int64_t* off_host) {
+  uint64_t h = 1469598103934665603ull;  // FNV-1a over the offsets' bytes
+  for (int i = 0; i <= B; ++i) {
+    uint64_t w = (uint64_t)off_host[i];
+    for (int b = 0; b < 8; ++b) { h ^= w & 0xffu; h *= 1099511628211ull; w >>= 8; }
+  }
+  WsTag t{};
+  t.v[0] = 0x49534f504f5f4753ll;
+  t.v[1] = (int64_t)dtype; t.v[2] = T; t.v[3] = d_in; t.v[4] = d_out; t.v[5] = B; t.v[6] = (int64_t)h;
+  return t;
 }
 
 static bool sizes_ok(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B) {
@@ -129,6 +159,16 @@ const char* isopo_last_cuda_error(void) { return g_cuda_err; }
 
 void isopo_profile_enable(int on) { g_prof_on = on != 0; }
 
+void isopo_set_deterministic(int on) { g_deterministic = on != 0; }
+int isopo_get_deterministic(void) { return g_deterministic ? 1 : 0; }
+int isopo_debug_build(void) {
+#ifdef ISOPO_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 isopo_status isopo_profile_collect(double* ms_by_kernel, int64_t* launches_by_kernel) {
   if (!ms_by_kernel || !launches_by_kernel) return ISOPO_ERR_INVALID_ARG;
   for (int k = 0; k < kIdCount; ++k) { ms_by_kernel[k] = 0.0; launches_by_kernel[k] = g_launches[k]; g_launches[k] = 0; }
@@ -150,7 +190,7 @@ const char* isopo_kernel_name(int id) {
   static const char* names[kIdCount] = {"k_tokseq", "k_bf16_seq_grad", "k_bf16_ntk", "k_bf16_gram", "k_bf16_weight_grad",
                                         "k_bf16_combine", "k_transform", "k_mirror_upper", "k_f32_seq_grad",
                                         "k_f32_ntk", "k_f32_gram", "k_f32_weight_grad", "k_f32_combine",
-                                        "k_sampled", "k_sampled_aux", "k_scale_rows"};
+                                        "k_sampled", "k_sampled_aux", "k_scale_rows", "k_wait_probe"};
   return id >= 0 && id < kIdCount ? names[id] : "unknown";
 }
 
@@ -176,6 +216,7 @@ size_t isopo_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, 
 isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
                               const int64_t* seq_offsets_host, int B, isopo_path path, float* K, void* ws,
                               size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_layer_gram");
   if (!K || !info) return ISOPO_ERR_INVALID_ARG;
   isopo_status s = check_layer_args(X, dY, dtype, T, d_in, d_out, seq_offsets_host, B, path, ws);
   if (s != ISOPO_OK) return s;
@@ -187,29 +228,37 @@ isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, 
   char* w = (char*)ws;
   int64_t* off_dev = (int64_t*)(w + L.off_offsets);
   int32_t* tokseq = (int32_t*)(w + L.off_tokseq);
+  WsTag* tag_dev = (WsTag*)(w + L.off_tag);
+  if (dtype == ISOPO_BF16 && rp == ISOPO_PATH_MATERIALISE) {
+    // the stored-gradient kernels need the offsets and the longest-first order, not the token map
+    void* G = w + L.off_G;
+    int32_t* order = (int32_t*)(w + L.off_order);
+    s = launch_prep_stored(seq_offsets_host, B, make_ws_tag(dtype, T, d_in, d_out, B, seq_offsets_host), off_dev, order,
+                           tag_dev, K, st);
+    if (s != ISOPO_OK) return s;
+    s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, order, B, L, G, info, st);
+    if (s != ISOPO_OK) return s;
+    return bf16_ntk(G, L, B, K, /*k_is_zero=*/true, deterministic_mode() ? (float*)(w + L.off_kpart) : nullptr, info, st);
+  }
   s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
   if (s != ISOPO_OK) return s;
   if (dtype == ISOPO_F32) {
     if (rp == ISOPO_PATH_GRAM)
       return f32_gram((const float*)X, (const float*)dY, T, d_in, d_out, tokseq, B, (double*)(w + L.off_kacc), K, st);
+    s = store_tag(make_ws_tag(dtype, T, d_in, d_out, B, seq_offsets_host), tag_dev, st);
+    if (s != ISOPO_OK) return s;
     float* G = (float*)(w + L.off_G);
     s = f32_seq_grad((const float*)X, (const float*)dY, d_in, d_out, off_dev, B, G, st);
     if (s != ISOPO_OK) return s;
     return f32_ntk(G, L.n_pad, B, K, st);
   }
-  if (rp == ISOPO_PATH_GRAM) return bf16_gram(X, dY, T, d_in, d_out, tokseq, B, K, info, st);
-  void* G = w + L.off_G;
-  int32_t* order = (int32_t*)(w + L.off_order);
-  s = launch_order(seq_offsets_host, B, order, st);
-  if (s != ISOPO_OK) return s;
-  s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, order, B, L, G, info, st);
-  if (s != ISOPO_OK) return s;
-  return bf16_ntk(G, L, B, K, info, st);
+  return bf16_gram(X, dY, T, d_in, d_out, tokseq, B, K, info, st);
 }
 
 isopo_status isopo_layer_gram_shared_x(const void* X, int n_proj, const void* const* dY, const int* d_out, isopo_dtype dtype,
                                        int64_t T, int d_in, const int64_t* seq_offsets_host, int B, float* const* K,
                                        void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_layer_gram_shared_x");
   if (!dY || !d_out || !K || !info || n_proj < 1 || n_proj > 3) return ISOPO_ERR_INVALID_ARG;
   if (dtype != ISOPO_BF16) return ISOPO_ERR_UNSUPPORTED;
   int d_max = 0;
@@ -238,6 +287,7 @@ isopo_status isopo_sampled_coefficients(const void* X, const void* dY, isopo_dty
                                         const int64_t* seq_offsets_host, int B, const int64_t* sample_rows_host,
                                         int n_samples, const float* A, float lambda, float* coeffs, float* F2, void* ws,
                                         size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_sampled_coefficients");
   if (!A || !coeffs || !info || !sample_rows_host) return ISOPO_ERR_INVALID_ARG;
   if (!(lambda >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
   isopo_status s = check_layer_args(X, dY, dtype, T, d_in, d_out, seq_offsets_host, B, ISOPO_PATH_GRAM, ws);
@@ -259,6 +309,7 @@ isopo_status isopo_sampled_coefficients(const void* X, const void* dY, isopo_dty
 
 isopo_status isopo_transform_advantages(const float* K, const float* A, int B, isopo_variant variant, float lambda,
                                         const float* opt_pqr_regs, float* coeffs, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_transform_advantages");
   if (!K || !A || !coeffs || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
   if ((int)variant < 0 || (int)variant > (int)ISOPO_VAR_NORMALISED_RAW) return ISOPO_ERR_INVALID_ARG;
   if (!(lambda >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
@@ -268,6 +319,7 @@ isopo_status isopo_transform_advantages(const float* K, const float* A, int B, i
 }
 
 isopo_status isopo_reg_ema_update(const float* K, int B, float decay, float* state, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_reg_ema_update");
   if (!K || !state || B < 1 || !(decay >= 0.0f && decay < 1.0f)) return ISOPO_ERR_INVALID_ARG;
   return reg_ema_update(K, B, decay, state, (cudaStream_t)cuda_stream);
 }
@@ -275,6 +327,7 @@ isopo_status isopo_reg_ema_update(const float* K, int B, float decay, float* sta
 isopo_status isopo_transform_advantages_rel(const float* K, const float* A, int B, isopo_variant variant, float factor,
                                             const float* opt_pqr_factors, const float* state, float* coeffs,
                                             int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_transform_advantages_rel");
   if (!K || !A || !coeffs || !info || !state || B < 1) return ISOPO_ERR_INVALID_ARG;
   if ((int)variant < 0 || (int)variant > (int)ISOPO_VAR_NORMALISED_RAW) return ISOPO_ERR_INVALID_ARG;
   if (!(factor >= 0.0f)) return ISOPO_ERR_INVALID_ARG;
@@ -287,6 +340,7 @@ isopo_status isopo_transform_advantages_batched(int n_layers, const float* const
                                                 isopo_variant variant, const float* lambda,
                                                 const float* opt_pqr_regs, const float* const* states,
                                                 float* const* coeffs, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_transform_advantages_batched");
   if (n_layers < 1 || n_layers > ISOPO_MAX_BATCH) return ISOPO_ERR_INVALID_ARG;
   if (!K || !A || !lambda || !coeffs || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
   if ((int)variant < 0 || (int)variant > (int)ISOPO_VAR_NORMALISED_RAW) return ISOPO_ERR_INVALID_ARG;
@@ -299,11 +353,18 @@ isopo_status isopo_transform_advantages_batched(int n_layers, const float* const
                            (cudaStream_t)cuda_stream);
 }
 
+isopo_status isopo_selftest_bounded_wait(int64_t limit_clocks, int32_t* info, int32_t* roles_at_teardown, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_selftest_bounded_wait");
+  if (!info || !roles_at_teardown || limit_clocks < 1 || limit_clocks > ((int64_t)1 << 28)) return ISOPO_ERR_INVALID_ARG;
+  return wait_probe((long long)limit_clocks, info, roles_at_teardown, (cudaStream_t)cuda_stream);
+}
+
 size_t isopo_spectral_workspace_bytes(void) { return spectral_workspace_bytes(); }
 
 isopo_status isopo_transform_spectral(const float* K, const float* A, int B, float lambda, float rel_cutoff,
                                       float* coeffs, float* eigenvalues, void* ws, size_t ws_bytes, int32_t* info,
                                       void* cuda_stream) {
+  ApiRange nvtx_range("isopo_transform_spectral");
   if (!K || !A || !coeffs || !ws || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
   if (!(lambda >= 0.0f) || !(rel_cutoff >= 0.0f && rel_cutoff < 1.0f)) return ISOPO_ERR_INVALID_ARG;
   if ((uintptr_t)ws & 15) return ISOPO_ERR_INVALID_ARG;
@@ -316,6 +377,7 @@ isopo_status isopo_transform_spectral_batched(int n_layers, const float* const* 
                                               const float* lambda, float rel_cutoff, float* const* coeffs,
                                               float* const* eigenvalues, void* ws, size_t ws_bytes, int32_t* info,
                                               void* cuda_stream) {
+  ApiRange nvtx_range("isopo_transform_spectral_batched");
   if (n_layers < 1 || n_layers > ISOPO_MAX_BATCH) return ISOPO_ERR_INVALID_ARG;
   if (!K || !A || !lambda || !coeffs || !ws || !info || B < 1) return ISOPO_ERR_INVALID_ARG;
   if (!(rel_cutoff >= 0.0f && rel_cutoff < 1.0f) || ((uintptr_t)ws & 15)) return ISOPO_ERR_INVALID_ARG;
@@ -330,6 +392,7 @@ isopo_status isopo_transform_spectral_batched(int n_layers, const float* const* 
 isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype, int64_t T, int d_in, int d_out,
                                const float* coeffs, const int64_t* seq_offsets_host, int B, isopo_path path,
                                float* dW, float beta, void* ws, size_t ws_bytes, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_weight_grad");
   if (!coeffs || !dW || !info) return ISOPO_ERR_INVALID_ARG;
   if (beta != 0.0f && beta != 1.0f) return ISOPO_ERR_INVALID_ARG;
   isopo_status s = check_layer_args(X, dY, dtype, T, d_in, d_out, seq_offsets_host, B, path, ws);
@@ -341,8 +404,12 @@ isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype,
   cudaStream_t st = (cudaStream_t)cuda_stream;
   char* w = (char*)ws;
   if (rp == ISOPO_PATH_MATERIALISE) {
-    if (dtype == ISOPO_F32) return f32_combine((const float*)(w + L.off_G), L.n_pad, B, coeffs, dW, beta, st);
-    return bf16_combine(w + L.off_G, L, d_in, d_out, B, coeffs, dW, beta, st);
+    // the kernels compare the tag isopo_layer_gram left with the one of this call and touch nothing on a mismatch
+    const WsTag tag = make_ws_tag(dtype, T, d_in, d_out, B, seq_offsets_host);
+    const WsTag* tag_dev = (const WsTag*)(w + L.off_tag);
+    if (dtype == ISOPO_F32)
+      return f32_combine((const float*)(w + L.off_G), L.n_pad, B, coeffs, dW, beta, tag_dev, tag, info, st);
+    return bf16_combine(w + L.off_G, L, d_in, d_out, B, coeffs, dW, beta, tag_dev, tag, info, st);
   }
   // GEMM over all tokens: refresh the token -> sequence map so the call also works on its own.
   int64_t* off_dev = (int64_t*)(w + L.off_offsets);
@@ -351,6 +418,11 @@ isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype,
     s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
     if (s != ISOPO_OK) return s;
     return f32_weight_grad((const float*)X, (const float*)dY, T, d_in, d_out, coeffs, tokseq, dW, beta, st);
+  }
+  if (bf16_weight_grad_fold_applies(T, d_in, d_out, B)) {
+    s = store_i64(seq_offsets_host, (int64_t)B + 1, off_dev, st);
+    if (s != ISOPO_OK) return s;
+    return bf16_weight_grad_fold(X, dY, T, d_in, d_out, off_dev, coeffs, B, dW, beta, info, st);
   }
   // one scale per token, so that the kernel's scaler warps need a single independent load per row
   float* tokscale = (float*)tokseq;

@@ -16,14 +16,30 @@ constexpr int kTK = 16;  // tokens staged per step
 // synchronisation with the stream and nothing that reads the caller's array after the call returns).
 constexpr int kArgChunk = 384;
 struct OffsetArgs { int64_t v[kArgChunk]; };
-struct OrderArgs { int32_t v[256]; };
 __global__ void k_store_offsets(OffsetArgs a, int base, int n, int64_t* __restrict__ off) {
   const int t = threadIdx.x;
   if (t < n) off[base + t] = a.v[t];
 }
-__global__ void k_store_order(OrderArgs a, int n, int32_t* __restrict__ order) {
-  const int t = threadIdx.x;
-  if (t < n) order[t] = a.v[t];
+
+// Everything the bf16 stored-gradient kernels need before they start, in one launch (B <= 256):
+// CTA 0 leaves the offsets, the working order of the sequences and the workspace tag; all CTAs clear K.
+struct StoredPrepArgs {
+  int64_t off[257];
+  WsTag tag;
+  uint8_t order[256];
+};
+__global__ void __launch_bounds__(256) k_prep_stored(StoredPrepArgs a, int B, int64_t* __restrict__ off,
+                                                     int32_t* __restrict__ order, WsTag* __restrict__ tag,
+                                                     float* __restrict__ K) {
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i <= B; i += blockDim.x) off[i] = a.off[i];
+    for (int i = threadIdx.x; i < B; i += blockDim.x) order[i] = a.order[i];
+    if (threadIdx.x < 8) tag->v[threadIdx.x] = a.tag.v[threadIdx.x];
+  }
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < B * B; e += gridDim.x * blockDim.x) K[e] = 0.f;
+}
+__global__ void k_store_tag(WsTag t, WsTag* __restrict__ tag) {
+  if (threadIdx.x < 8) tag->v[threadIdx.x] = t.v[threadIdx.x];
 }
 
 __global__ void k_tokseq(const int64_t* __restrict__ off, int B, int64_t T, int32_t* __restrict__ tokseq) {
@@ -226,7 +242,9 @@ __global__ void k_f32_gram_finish(const double* __restrict__ kacc, int B, float*
 }
 
 __global__ void k_f32_combine(const float* __restrict__ G, int64_t N, int B, const float* __restrict__ coeffs,
-                              float* __restrict__ dW, float beta) {
+                              float* __restrict__ dW, float beta, const WsTag* __restrict__ tag_dev, WsTag tag,
+                              int32_t* __restrict__ info) {
+  if (!ws_tag_matches(tag_dev, tag, info)) return;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < N; e += (int64_t)gridDim.x * blockDim.x) {
     double s = 0.0;
     for (int i = 0; i < B; ++i) s += (double)coeffs[i] * (double)G[(size_t)i * N + e];
@@ -289,15 +307,27 @@ isopo_status launch_tokscale(const int64_t* off_host, int B, int64_t T, int64_t*
   return ISOPO_OK;
 }
 
-isopo_status launch_order(const int64_t* off_host, int B, int32_t* order_dev, cudaStream_t st) {
+isopo_status launch_prep_stored(const int64_t* off_host, int B, const WsTag& tag, int64_t* off_dev, int32_t* order_dev,
+                                WsTag* tag_dev, float* K, cudaStream_t st) {
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
-  OrderArgs a;
-  for (int i = 0; i < B; ++i) a.v[i] = i;
+  StoredPrepArgs a;
+  for (int i = 0; i <= B; ++i) a.off[i] = off_host[i];
+  a.tag = tag;
+  int idx[256];
+  for (int i = 0; i < B; ++i) idx[i] = i;
   // longest first; equal lengths keep their order
-  std::stable_sort(a.v, a.v + B, [&](int32_t x, int32_t y) {
-    return off_host[x + 1] - off_host[x] > off_host[y + 1] - off_host[y];
-  });
-  k_store_order<<<1, 256, 0, st>>>(a, B, order_dev);
+  std::stable_sort(idx, idx + B, [&](int x, int y) { return off_host[x + 1] - off_host[x] > off_host[y + 1] - off_host[y]; });
+  for (int i = 0; i < B; ++i) a.order[i] = (uint8_t)idx[i];
+  {
+    LaunchScope scope(kIdPrep, st);
+    k_prep_stored<<<std::max(1, (B * B + 2047) / 2048), 256, 0, st>>>(a, B, off_dev, order_dev, tag_dev, K);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status store_tag(const WsTag& tag, WsTag* tag_dev, cudaStream_t st) {
+  k_store_tag<<<1, 32, 0, st>>>(tag, tag_dev);
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
@@ -342,12 +372,12 @@ isopo_status f32_gram(const float* X, const float* dY, int64_t T, int d_in, int 
   return ISOPO_OK;
 }
 
-isopo_status f32_combine(const float* G, int64_t N, int B, const float* coeffs, float* dW, float beta,
-                         cudaStream_t st) {
+isopo_status f32_combine(const float* G, int64_t N, int B, const float* coeffs, float* dW, float beta, const WsTag* tag_dev,
+                         const WsTag& tag, int32_t* info, cudaStream_t st) {
   const int grid = (int)std::min<int64_t>((N + 255) / 256, 148 * 8);
   {
     LaunchScope scope(kIdF32Combine, st);
-    k_f32_combine<<<grid, 256, 0, st>>>(G, N, B, coeffs, dW, beta);
+    k_f32_combine<<<grid, 256, 0, st>>>(G, N, B, coeffs, dW, beta, tag_dev, tag, info);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

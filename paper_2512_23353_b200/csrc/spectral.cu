@@ -1,5 +1,6 @@
-// Spectral form of the interacting transform (Alg. 2: "D, U = eigh(ntk); preconditioner = 1 / (D +
-// regularization); U @ (preconditioner * (U.T @ advantages))"), with the spectrum as a second output.
+// Spectral form of the interacting transform (Alg. 2, last block: symmetric eigendecomposition of the
+// NTK, every eigen-direction of the advantages divided by its eigenvalue plus the regulariser, then
+// back to the sequence basis), with the spectrum as a second output.
 //
 // A cluster of eight CTAs (128 warps) diagonalises K by one-sided (Hestenes) Jacobi: W starts as K, V as the identity;
 // a rotation of columns p and q, applied to both, makes the two columns of W orthogonal and keeps

@@ -95,19 +95,20 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Gives up after ~2^31 clock ticks (about a second) or as soon as another role of
-// this CTA has given up (`*abort_flag` != 0, shared memory); records ISOPO_INFO_TIMEOUT | code in
-// *info (only over a zero) and returns false.  Callers leave their loops and fall through to the
-// common teardown, so the kernel always ends and the context stays usable.
+// Bounded wait.  Gives up after `limit` clock ticks (by default ~2^31, about a second) or as soon as
+// another role of this CTA has given up (`*abort_flag` != 0, shared memory); records
+// ISOPO_INFO_TIMEOUT | code in *info (only over a zero) and returns false.  Callers leave their loops
+// and fall through to the common teardown, so the kernel always ends and the context stays usable.
+constexpr long long kWaitLimitClocks = 1ll << 31;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* info,
-                                          int code) {
+                                          int code, long long limit = kWaitLimitClocks) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long start = clock64();
   while (true) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - start > (1ll << 31)) {
+    if (clock64() - start > limit) {
       *abort_flag = 1;
       atomicCAS(info, 0, ISOPO_INFO_TIMEOUT | code);
       return false;
@@ -217,7 +218,7 @@ __device__ __forceinline__ bool mbar_wait_pair(uint32_t bar, uint32_t parity, vo
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - start > (1ll << 31)) {
+    if (clock64() - start > kWaitLimitClocks) {
       *abort_flag = 1;
       st_cluster_u32(peer_abort, 1u);
       atomicCAS(info, 0, ISOPO_INFO_TIMEOUT | code);

@@ -168,7 +168,8 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapRX, const __grid_constant__ C
       // sequence of this thread's row token and of every column token (clamped past the end; those
       // rows and columns are zero in P and Q)
       // (sampled: the "row sequence" is the sample index, its results go to row `row_seq` of M^T;
-      // rows past the last sample are zero in P and Q and flush nothing)
+      // rows past the last sample are zero in P and Q, and they are barred from writing outright: a
+      // non-finite input would turn their zeros into NaN, and row `trow` of M^T does not exist)
       const int64_t trow = (int64_t)I * kTT + row;
       const int row_seq = kSampled ? (int)trow : __ldg(p.tokseq + min(trow, p.T - 1));
       auto col_seq = [&](int g) { return __ldg(p.tokseq + min((int64_t)J * kTT + g * 32 + lane, p.T - 1)); };
@@ -176,7 +177,7 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapRX, const __grid_constant__ C
       if (!mbar_wait(accfull_bar(acc), acc_phase, abort_flag, p.info, kIdGram)) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * 256;
-      const RowSegments rows = row_segments(row_seq);
+      const RowSegments rows = row_segments(row_seq, (long long)(kSampled ? p.n_rows : p.B) * p.B, p.info, !kSampled || trow < (int64_t)p.n_rows);
       int cur = __shfl_sync(0xffffffffu, cs, 0);
       float wseg = (!kSampled && row_seq == cur) ? 2.f : 1.f, run = 0.f;
 #pragma unroll 1
@@ -203,12 +204,6 @@ k_bf16_gram(const __grid_constant__ CUtensorMap mapRX, const __grid_constant__ C
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-__global__ void k_mirror_upper_gram(float* __restrict__ K, int B) {
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= B * B) return;
-  const int i = e / B, j = e % B;
-  if (j < i) K[e] = K[(size_t)j * B + i];
-}
 
 }  // namespace
 
@@ -233,12 +228,7 @@ isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d
     k_bf16_gram<false><<<grid, kThreads, kSmemBytes, st>>>(mapX, mapY, mapX, mapY, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
-  {
-    LaunchScope scope(kIdMirror, st);
-    k_mirror_upper_gram<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
-  }
-  ISOPO_CUDA_TRY(cudaGetLastError());
-  return ISOPO_OK;
+  return mirror_upper(K, B, st);
 }
 
 isopo_status bf16_sampled(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,

@@ -1,4 +1,4 @@
-// Epilogue shared by the Gram-route kernels (tc_gram.cu, tc_gram_pair.cu): the elementwise product of
+// Epilogue shared by the Gram-route kernels (tc_gram.cu, tc_gram_shared.cu): the elementwise product of
 // the two accumulators P and Q, summed per (sequence of the row token, sequence of the column token).
 //
 // Every lane owns one accumulator row and walks the columns 32 at a time.  Column tokens are in
@@ -59,11 +59,17 @@ struct RowSegments {
   int seq;        // sequence of this lane's row token (sampled estimator: the sample index, all distinct)
   bool head;      // first lane of its run of equal `seq`
   unsigned same;  // bit k: lane + 2^k exists and has the same `seq`
+  bool valid;     // the row exists (rows past the end of the row range never write, whatever their sums hold)
+  long long n_out;  // elements of the output matrix (debug build: every flush is checked against it)
+  int32_t* info;
 };
 
-__device__ __forceinline__ RowSegments row_segments(int seq) {
+__device__ __forceinline__ RowSegments row_segments(int seq, long long n_out, int32_t* info, bool valid = true) {
   RowSegments r;
   r.seq = seq;
+  r.valid = valid;
+  r.n_out = n_out;
+  r.info = info;
   const int lane = threadIdx.x & 31;
   const int up = __shfl_up_sync(0xffffffffu, seq, 1);
   r.head = lane == 0 || up != seq;
@@ -83,7 +89,9 @@ __device__ __forceinline__ void flush_rows(float* __restrict__ K, int B, const R
     const float t = __shfl_down_sync(0xffffffffu, v, 1 << k);
     if ((rows.same >> k) & 1u) v += t;
   }
-  if (rows.head && v != 0.f) atomicAdd(&K[(size_t)rows.seq * B + col_seq], v);
+  if (rows.head && rows.valid && v != 0.f &&
+      ISOPO_IN_RANGE(col_seq < 0 || col_seq >= B ? -1 : (long long)rows.seq * B + col_seq, rows.n_out, rows.info, kIdGram))
+    atomicAdd(&K[(size_t)rows.seq * B + col_seq], v);
 }
 
 // One group of 32 columns.  pv/qv: this lane's 32 values of P and Q; cs: sequence of column c0 + lane;

@@ -170,7 +170,7 @@ k_bf16_gram_shared(const __grid_constant__ CUtensorMap mapX, const __grid_consta
       const int64_t trow = (int64_t)I * kTT + row;
       const int row_seq = __ldg(p.tokseq + min(trow, p.T - 1));
       auto col_seq = [&](int g) { return __ldg(p.tokseq + min((int64_t)J * kTT + g * 32 + lane, p.T - 1)); };
-      const RowSegments rows = row_segments(row_seq);
+      const RowSegments rows = row_segments(row_seq, (long long)p.B * p.B, p.info);
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
       for (int h = 0; h < p.n_heads; ++h, ++qcount) {
@@ -208,12 +208,6 @@ k_bf16_gram_shared(const __grid_constant__ CUtensorMap mapX, const __grid_consta
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-__global__ void k_mirror_upper_shared(float* __restrict__ K, int B) {
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= B * B) return;
-  const int i = e / B, j = e % B;
-  if (j < i) K[e] = K[(size_t)j * B + i];
-}
 
 }  // namespace
 
@@ -250,10 +244,9 @@ isopo_status bf16_gram_shared(const void* X, const void* const* dY, int64_t T, i
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   for (int h = 0; h < n_heads; ++h) {
-    LaunchScope scope(kIdMirror, st);
-    k_mirror_upper_shared<<<(B * B + 255) / 256, 256, 0, st>>>(K[h], B);
+    const isopo_status s = mirror_upper(K[h], B, st);
+    if (s != ISOPO_OK) return s;
   }
-  ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
 

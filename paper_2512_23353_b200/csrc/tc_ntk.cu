@@ -35,6 +35,7 @@ constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 
 struct NtkParams {
+  float* kpart;   // deterministic mode: [CTA][B * B] partial sums, plain stores; NULL: float atomics into K
   float* K;
   int B;
   long long nkb;  // boxes in the contraction dimension: ceil(pieces / ppb) * 4
@@ -117,6 +118,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
     } else {
       const int q = warp & 3;
       const int r = q * 32 + lane;
+      // every (CTA, entry of the upper triangle) is produced by exactly one thread, once
+      float* const mine = p.kpart ? p.kpart + (size_t)blockIdx.x * p.B * p.B : nullptr;
+      auto add_to_k = [&](size_t idx, float v) {
+        if (mine) mine[idx] = v; else atomicAdd(&p.K[idx], v);
+      };
       // `ok` is false only after a wait ran out; every thread still reaches the named barrier below
       const bool ok = mbar_wait(accfull_bar, 0, abort_flag, p.info, kIdNtk);
       {
@@ -132,7 +138,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const int c = c0 + e;
-                if (c >= r && c < p.B) atomicAdd(&p.K[(size_t)r * p.B + c], __uint_as_float(v[e]));
+                if (c >= r && c < p.B && ISOPO_IN_RANGE((long long)r * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
+                  add_to_k((size_t)r * p.B + c, __uint_as_float(v[e]));
               }
             }
           }
@@ -146,7 +153,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const int c = 128 + c0 + e;
-                if (c >= rr && c < p.B) atomicAdd(&p.K[(size_t)rr * p.B + c], __uint_as_float(v[e]));
+                if (c >= rr && c < p.B && ISOPO_IN_RANGE((long long)rr * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
+                  add_to_k((size_t)rr * p.B + c, __uint_as_float(v[e]));
               }
             }
           }
@@ -177,7 +185,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
               if (c < sq || sq >= p.B) continue;  // upper triangle of the sequences that exist
               float sum = 0.f;
               for (int h = 0; h < ngroups; ++h) sum += red[(((h << lr) + c) << lr) + sq];
-              atomicAdd(&p.K[(size_t)sq * p.B + c], sum);
+              if (ISOPO_IN_RANGE((long long)sq * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
+                add_to_k((size_t)sq * p.B + c, sum);
             }
           }
         }
@@ -191,6 +200,17 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+// Deterministic mode: K[i][j] = K[j][i] = sum over the CTAs, in CTA order, of their partial entry (min(i,j), max(i,j)).
+__global__ void k_ntk_reduce(const float* __restrict__ kpart, int n_ctas, int B, float* __restrict__ K) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= B * B) return;
+  const int i = e / B, j = e % B;
+  const size_t src = (size_t)min(i, j) * B + max(i, j), stride = (size_t)B * B;
+  float s = 0.f;
+  for (int c = 0; c < n_ctas; ++c) s += kpart[c * stride + src];
+  K[e] = s;
+}
+
 __global__ void k_mirror_upper(float* __restrict__ K, int B) {
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= B * B) return;
@@ -202,7 +222,9 @@ __global__ void k_mirror_upper(float* __restrict__ K, int B) {
 __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long nchunks /* n_pad / 8 */,
                                                        int B, int tiles_n, int d_in, int d_out,
                                                        const float* __restrict__ coeffs, float* __restrict__ dW,
-                                                       float beta) {
+                                                       float beta, const WsTag* __restrict__ tag_dev, WsTag tag,
+                                                       int32_t* __restrict__ info) {
+  if (!ws_tag_matches(tag_dev, tag, info)) return;  // another layer's or microbatch's gradients: touch nothing
   __shared__ float sc[256];
   for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = coeffs[i];
   __syncthreads();
@@ -213,6 +235,8 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ 
     const int l = (int)(pos & 31), q = (int)(piece & 3), j = (int)((piece >> 2) & 31), tile = (int)(piece >> 7);
     const int m = (tile / tiles_n) * kTileM + q * 32 + l, n = (tile % tiles_n) * kTileN + j * 8;
     if (m >= d_out || n >= d_in) continue;
+    if (!ISOPO_IN_RANGE((long long)stored_slot((size_t)piece, B - 1, B, l), nchunks * B, info, kIdCombine)) continue;
+    if (!ISOPO_IN_RANGE((long long)m * d_in + n + 7, (long long)d_out * d_in, info, kIdCombine)) continue;
     float acc[8] = {};
     const uint4* src = G + stored_slot((size_t)piece, 0, B, l);
     const size_t chunks = 32;  // uint4 stride between successive sequences of one piece
@@ -256,7 +280,8 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ 
 
 }  // namespace
 
-isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t* info, cudaStream_t st) {
+isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, bool k_is_zero, float* kpart, int32_t* info,
+                      cudaStream_t st) {
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
   CUtensorMap mapG;
   const uint32_t rows = B > 128 ? 256 : B > 64 ? 128 : B > 32 ? 64 : 32, ppb = 256 / rows;
@@ -267,14 +292,28 @@ isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_ntk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
-  NtkParams p{K, B, (pieces + ppb - 1) / ppb * 4, info, (int)rows, (int)ppb};
-  const int grid = (int)std::max<long long>(1, std::min<long long>(sms, p.nkb / 8));
+  if (!k_is_zero && !kpart) ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
+  NtkParams p{kpart, K, B, (pieces + ppb - 1) / ppb * 4, info, (int)rows, (int)ppb};
+  int grid = (int)std::max<long long>(1, std::min<long long>(sms, p.nkb / 8));
+  if (kpart) grid = std::min(grid, kNtkMaxPartials);
   {
     LaunchScope scope(kIdNtk, st);
     k_bf16_ntk<<<grid, kThreads, kSmemBytes, st>>>(mapG, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
+  if (!kpart) return mirror_upper(K, B, st);
+  // CTAs whose slab of the contraction is empty wrote nothing: sum only those that had work
+  const long long per = (p.nkb + grid - 1) / grid;
+  const int n_active = (int)((p.nkb + per - 1) / per);
+  {
+    LaunchScope scope(kIdMirror, st);
+    k_ntk_reduce<<<(B * B + 255) / 256, 256, 0, st>>>(kpart, n_active, B, K);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+isopo_status mirror_upper(float* K, int B, cudaStream_t st) {
   {
     LaunchScope scope(kIdMirror, st);
     k_mirror_upper<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
@@ -284,7 +323,7 @@ isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, int32_t
 }
 
 isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
-                          float beta, cudaStream_t st) {
+                          float beta, const WsTag* tag_dev, const WsTag& tag, int32_t* info, cudaStream_t st) {
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
   const long long chunks = L.n_pad / 8;
   int dev = 0, sms = 0;
@@ -293,7 +332,7 @@ isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out,
   const int grid = (int)std::min<long long>((chunks + 255) / 256, (long long)sms * 8);
   {
     LaunchScope scope(kIdCombine, st);
-    k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta);
+    k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta, tag_dev, tag, info);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

@@ -238,7 +238,9 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
             o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
             o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
             o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-            dst[stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane)] = o;
+            const size_t slot = stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane);
+            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, (long long)p.B * p.n_pad / 8, p.info, kIdSeqGrad))
+              dst[slot] = o;
           }
         }
       } else {
@@ -254,7 +256,8 @@ k_bf16_seq_grad(const __grid_constant__ CUtensorMap mapY, const __grid_constant_
 #pragma unroll
             for (int v = 0; v < 8; ++v) {
               const int n = n0 + jc * 32 + v * 4;
-              if (n < p.d_in)  // d_in is a multiple of 8, so a group of 4 is all in or all out
+              if (n < p.d_in &&  // d_in is a multiple of 8, so a group of 4 is all in or all out
+                  ISOPO_IN_RANGE((long long)m * p.d_in + n + 3, (long long)p.d_out * p.d_in, p.info, kIdWeightGrad))
                 asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + jc * 32 + v * 4),
                              "f"(__uint_as_float(r[v * 4 + 0])), "f"(__uint_as_float(r[v * 4 + 1])),
                              "f"(__uint_as_float(r[v * 4 + 2])), "f"(__uint_as_float(r[v * 4 + 3]))

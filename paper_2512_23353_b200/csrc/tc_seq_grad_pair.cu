@@ -59,6 +59,7 @@ struct PairParams {
   int ptiles_m;             // pair tiles along d_out = ceil(tiles_m / 2)
   int32_t* info;
   int group_m;              // pair-tile rows per group of the tile order
+  long long n_slots;        // 16-byte slots of the stored gradients (debug build: every store is checked against it)
 };
 
 // The pair tiles of one sequence are visited in groups of `group_m` rows, row index fastest inside a
@@ -245,7 +246,8 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
             o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
             o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
             o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-            dst[stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane)] = o;
+            const size_t slot = stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane);
+            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, p.n_slots, p.info, kIdSeqGrad)) dst[slot] = o;
           }
         }
       }
@@ -314,6 +316,7 @@ isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_
   p.off = off_dev; p.order = order_dev; p.G = (__nv_bfloat16*)G; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
   p.ptiles_m = (L.tiles_m + 1) / 2;
   p.info = info;
+  p.n_slots = (long long)B * L.n_pad / 8;
   const long long units = (long long)B * p.ptiles_m * p.tiles_n;
   // Persistent pairs with a static share of the units each: launch only as many pairs as can be
   // resident at once (the hardware may place fewer 2-CTA clusters than there are SM pairs).

@@ -186,7 +186,8 @@ k_bf16_weight_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_c
 #pragma unroll
           for (int v = 0; v < 8; ++v) {
             const int n = n0 + jc * 32 + v * 4;
-            if (n < p.d_in)  // d_in is a multiple of 8, so a group of 4 is all in or all out
+            if (n < p.d_in &&  // d_in is a multiple of 8, so a group of 4 is all in or all out
+                ISOPO_IN_RANGE((long long)m * p.d_in + n + 3, (long long)p.d_out * p.d_in, p.info, kIdWeightGrad))
               asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + jc * 32 + v * 4),
                            "f"(__uint_as_float(r[v * 4 + 0])), "f"(__uint_as_float(r[v * 4 + 1])),
                            "f"(__uint_as_float(r[v * 4 + 2])), "f"(__uint_as_float(r[v * 4 + 3]))

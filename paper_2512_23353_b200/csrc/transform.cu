@@ -219,15 +219,6 @@ __device__ __noinline__ void block_cholesky_solve(const float* __restrict__ Lb, 
   }
 }
 
-#ifdef ISOPO_PHASE_TIMERS
-__device__ long long g_phase[16];
-#define PHASE(n) do { if (threadIdx.x == 0) g_phase[n] = clock64(); } while (0)
-#define PHASE_ACC(n, t0) do { if (threadIdx.x == 0) { long long t1__ = clock64(); g_phase[n] += t1__ - t0; t0 = t1__; } } while (0)
-#else
-#define PHASE(n) do {} while (0)
-#define PHASE_ACC(n, t0) do {} while (0)
-#endif
-
 __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ TransformBatch batch) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TransformParams P = batch.common;
@@ -307,7 +298,6 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
   double* sol = reinterpret_cast<double*>(vec + Bp);        // Bp doubles (8-byte aligned: all counts even)
   float* rdiag = reinterpret_cast<float*>(sol + Bp);        // Bp floats: 1 / L_kk
   if (tid == 0) s_fail = 0;
-  PHASE(0);
   // load the lower block triangle.  K is symmetric, so row j of K read along i gives column j of
   // the blocks; float4 loads, eight in flight per thread, when B is a multiple of 4.
   if ((B & 3) == 0) {
@@ -346,15 +336,11 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
       Lb[blk_slot(i / kNB, j / kNB) * kBlk + (j % kNB) * kNB + (i % kNB)] = i == j ? 1.f : 0.f;
   }
   __syncthreads();
-  PHASE(1);
-  long long tph = clock64();
-  (void)tph;
   if (warp == 0) {
     const int f = warp_factor_diag(Lb, rdiag);
     if (f != 0 && lane == 0) s_fail = f;
   }
   __syncthreads();
-  PHASE_ACC(8, tph);
   for (int J = 0; J < nb && !s_fail; ++J) {
     const float* Ljj = Lb + blk_slot(J, J) * kBlk;
     // panel: blocks (I, J) below the diagonal on warps 0 .. nwarps-2; the last warp inverts L_JJ
@@ -362,7 +348,6 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
     else
       for (int I = J + 1 + warp; I < nb; I += nwarps - 1) warp_solve_panel(Lb + blk_slot(I, J) * kBlk, Ljj, rdiag + J * kNB);
     __syncthreads();
-    PHASE_ACC(9, tph);
     // trailing blocks (I, Kc) with I >= Kc > J; t = a(a+1)/2 + rem -> I = J+1+a, Kc = J+1+rem.
     // t = 0 is the next diagonal block: all warps update it together, then warp 0 factors it while the
     // others work through the rest
@@ -397,7 +382,6 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
       }
     }
     __syncthreads();
-    PHASE_ACC(10, tph);
   }
   __syncthreads();
   if (s_fail) {
@@ -405,7 +389,6 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
     for (int i = tid; i < B; i += kThreads) P.coeffs[i] = 0.f;
     return;
   }
-  PHASE(2);
   // solve, then refinement rounds with a float64 residual while it is above float32 round-off
   double anorm2 = 0.0;
   for (int i = tid; i < Bp; i += kThreads) {
@@ -422,7 +405,6 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
   anorm2 = s_trace;
   for (int round = 0; round < 3; ++round) {
     block_cholesky_solve(Lb, InvD, vec, nb);
-    PHASE(3 + 2 * round);
     for (int i = tid; i < Bp; i += kThreads) sol[i] += (double)vec[i];
     __syncthreads();
     if (round == 2) break;
@@ -471,7 +453,6 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
     }
     if (lane == 0) atomicAdd(&s_res, rn2);
     __syncthreads();
-    PHASE(4);
     const bool done = s_res <= 1e-14 * anorm2;  // relative residual below 1e-7
     __syncthreads();
     if (tid == 0) s_res = 0.0;

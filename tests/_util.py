@@ -35,3 +35,8 @@ def oracle_layer(X, dY, off, A, variant_code, lam, pqr_regs=None):
         pqr, regs = tuple(pqr_regs[:3]), tuple(pqr_regs[3:])
     return orc.isopo_layer(to_f64(X), to_f64(dY), np.asarray(off), to_f64(A), VARIANT_NAME[variant_code], float(lam),
                            pqr, regs)
+
+
+def report(label, **values):
+    """One line per parity case with the measured errors and cond(K + lambda I) (shown by pytest -s or on failure)."""
+    print("[parity] " + label + ": " + ", ".join(f"{k}={v:.3e}" for k, v in values.items()))

@@ -8,7 +8,7 @@ import pytest
 import torch
 
 from oracle import isopo_oracle as orc
-from tests._util import offdiag_rel_fro, oracle_layer, rel_fro, to_f64
+from tests._util import offdiag_rel_fro, oracle_layer, rel_fro, report, to_f64
 from paper_2512_23353_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -63,13 +63,18 @@ def test_layer_matches_oracle(b, path, case):
         assert np.array_equal(K, K.T)
         assert rel_fro(K, K_o) <= TOL, rel_fro(K, K_o)
         c_o = orc.transform_advantages(K_o, to_f64(A), orc.NORMALISED if variant == b.VAR_NORMALISED else orc.INTERACTING, lam)
-        cond = np.linalg.cond(K_o + lam * np.eye(B)) if variant == b.VAR_INTERACTING else 1.0
-        assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL * max(1.0, cond / 1e3), (variant, cond)
-        # dW against the oracle's dW for the GPU's own coefficients (isolates the GEMM / combine)
-        dW_o = orc.weight_gradient(G, to_f64(res.coeffs))
-        assert rel_fro(res.dW.cpu().numpy(), dW_o) <= TOL, rel_fro(res.dW.cpu().numpy(), dW_o)
-        if cond < 50:
-            assert rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)) <= TOL
+        cond = float(np.linalg.cond(K_o + lam * np.eye(B))) if variant == b.VAR_INTERACTING else 1.0
+        errs = dict(K=rel_fro(K, K_o), c=rel_fro(res.coeffs.cpu().numpy(), c_o),
+                    # dW for the library's own coefficients (isolates the GEMM / combine) and fully independent
+                    dW_own_c=rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, to_f64(res.coeffs))),
+                    dW=rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)), cond=cond)
+        report(f"case {case} {path} variant {variant}", **errs)
+        # These shapes are hand-built edge cases, half of them with correlated tokens: the solve amplifies
+        # the rounding of K by cond(K + lambda I), so the coefficients (and the dW that inherits them) are
+        # allowed tol * cond / 1e3 beyond cond = 1e3; everything else is held to the flat tolerance.
+        allow = TOL * max(1.0, cond / 1e3)
+        assert errs["c"] <= allow and errs["dW"] <= allow, errs
+        assert errs["dW_own_c"] <= TOL, errs
     if len(Ls) > 1 and case % 2 == 1:
         assert offdiag_rel_fro(K, K_o) <= TOL
 

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from tests._util import offdiag_rel_fro, oracle_layer, rel_fro
+from tests._util import report, offdiag_rel_fro, oracle_layer, rel_fro
 from paper_2512_23353_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -76,9 +76,14 @@ def test_edge_shapes(b, path, shape):
     for variant, lam in ((b.VAR_NORMALISED, 0.0), (b.VAR_INTERACTING, 0.5)):
         res, K_o, c_o, dW_o = _run(b, X, dY, off, A, variant, lam, pcode)
         assert res.info == 0
-        assert rel_fro(res.K.cpu().numpy(), K_o) <= TOL
-        assert rel_fro(res.coeffs.cpu().numpy(), c_o) <= TOL * max(1.0, np.linalg.cond(K_o + lam * np.eye(B)) / 100)
-        assert rel_fro(res.dW.cpu().numpy(), dW_o) <= TOL * max(1.0, np.linalg.cond(K_o + lam * np.eye(B)) / 100)
+        cond = float(np.linalg.cond(K_o + lam * np.eye(B)))
+        errs = dict(K=rel_fro(res.K.cpu().numpy(), K_o), c=rel_fro(res.coeffs.cpu().numpy(), c_o),
+                    dW=rel_fro(res.dW.cpu().numpy(), dW_o), cond=cond)
+        report(f"edge shape {shape} {path} variant {variant}", **errs)
+        # hand-built shapes (one sequence, single-token sequences): the float32 solve is allowed the
+        # amplification cond / 100 of K's rounding; K itself is held to the flat 1e-5
+        assert errs["K"] <= TOL
+        assert errs["c"] <= TOL * max(1.0, cond / 100) and errs["dW"] <= TOL * max(1.0, cond / 100), errs
     if Lmax == 1:
         Kh = (dY.astype(np.float64) @ dY.astype(np.float64).T) * (X.astype(np.float64) @ X.astype(np.float64).T)
         assert rel_fro(res.K.cpu().numpy(), Kh) <= TOL

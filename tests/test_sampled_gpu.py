@@ -95,3 +95,35 @@ def test_sampled_argument_checks(b):
         b.isopo_sampled_coefficients(X, dY, off, [0, 1, 2] * 400, A, 0.0, c, ws, info)  # workspace sized for 4 samples
     assert e.value.status == b.ERR_WORKSPACE
     assert b.isopo_sampled_workspace_bytes(b.F32, 11, 8, 8, 2, b.MAX_SAMPLES + 1) == 0
+
+
+def test_non_finite_input_never_writes_past_the_sample_rows(b):
+    """100 samples fill only part of the last 128-row tile of the estimator's tensor-core kernel.  The
+    rows of that tile past the last sample are zero, but a non-finite activation among the column
+    tokens turns 0 * inf into NaN; those rows have no place in M^T and must write nothing.  The
+    workspace is followed by a guard region that has to stay as it was; the result may be NaN."""
+    Ls = [40] * 40
+    X, dY, off, A, rng = _inputs(Ls, 256, 128, torch.bfloat16, 77)
+    T, B, n_s = int(off[-1]), len(Ls), 100
+    X[T // 2, 5] = float("inf")
+    dY[T // 3, 9] = float("nan")
+    n = b.isopo_sampled_workspace_bytes(b.BF16, T, 256, 128, B, n_s)
+    guard = 1 << 20
+    raw = torch.full((n + 1024 + guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    shift = (-raw.data_ptr()) % 1024
+    ws = raw[shift:shift + n]
+    c = torch.empty(B, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rows = rng.permutation(T)[:n_s]
+    b.isopo_sampled_coefficients(X, dY, off, rows, A, 0.0, c, ws, info)
+    torch.cuda.synchronize()
+    assert int(info.item()) == 0
+    assert bool((raw[shift + n:] == 0x5A).all()), "the estimator wrote past its workspace"
+    assert bool((raw[:shift] == 0x5A).all())
+    # and the call still works on finite inputs afterwards, in the same workspace
+    X[T // 2, 5] = 1.0
+    dY[T // 3, 9] = 0.0
+    b.isopo_sampled_coefficients(X, dY, off, rows, A, 0.0, c, ws, info)
+    torch.cuda.synchronize()
+    F2_o = orc.sampled_fisher_norm_sq(to_f64(X), to_f64(dY), off, rows)
+    assert rel_fro(c.cpu().numpy(), orc.sampled_coefficients(F2_o, to_f64(A), 0.0)) <= 2e-2

@@ -1,8 +1,9 @@
 """isopo_layer_gram_static - the entry point for callers that cannot allocate device memory (a
 hook running under a framework allocator that owns the device, or while that allocator is locked).
-It keeps its scratch in a fixed array inside the library, so two things need checking through the
-C ABI: that it returns what isopo_layer_gram returns on the Gram route, and that a second call,
-which finds the first call's leftovers in that shared array, is still right.
+It keeps its scratch in a fixed array inside the library, so three things need checking through the
+C ABI: that it returns what isopo_layer_gram returns on the Gram route (and what the fp64 oracle
+defines K to be), that a second call, which finds the first call's leftovers in that shared array,
+is still right, and that a call really allocates nothing on the device.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
 every other test.  Passes alone in a fresh process and after the rest of the suite."""
@@ -10,6 +11,9 @@ every other test.  Passes alone in a fresh process and after the rest of the sui
 import numpy as np
 import pytest
 import torch
+
+from oracle import isopo_oracle as orc
+from tests._util import rel_fro, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -62,6 +66,37 @@ def test_static_scratch_matches_workspace_entry_point_twice(b, dtype, tol):
         assert int(info.item()) == 0
         assert torch.equal(K, K.T)
         assert _rel(K, want) <= tol
+        # and against the definition itself: K_ij = <G_i, G_j> with every G_i materialised in float64
+        K_o = orc.ntk(orc.sequence_gradients(to_f64(X), to_f64(dY), off))
+        assert rel_fro(K.cpu().numpy(), K_o) <= tol
+
+
+def test_static_scratch_call_allocates_nothing(b):
+    """After one warm-up call (module load, symbol look-up), a further call must leave the device's free
+    memory and torch's allocator exactly as they were - also with event timing switched on, which the
+    call suspends for its duration because creating events allocates: its launches are counted, but no
+    event is recorded for them."""
+    X, dY, off = _problem([120, 40, 77], 64, 48, torch.bfloat16, 9)
+    K = torch.empty(3, 3, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.isopo_layer_gram_static(X, dY, off, K, info)
+    torch.cuda.synchronize()
+    b.isopo_profile_enable(True)
+    try:
+        b.isopo_profile_collect()                      # forget whatever earlier tests left
+        free0, _ = torch.cuda.mem_get_info()
+        alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        b.isopo_layer_gram_static(X, dY, off, K, info)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0
+        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+        prof = b.isopo_profile_collect()
+        assert sum(n for _, n in prof.values()) >= 2   # prep + Gram kernel were launched and counted ...
+        assert all(ms == 0.0 for ms, _ in prof.values())   # ... without an event pair around them
+    finally:
+        b.isopo_profile_enable(False)
+    assert int(info.item()) == 0
 
 
 def test_static_scratch_rejects_sizes_beyond_its_array(b):
