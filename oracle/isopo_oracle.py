@@ -97,26 +97,29 @@ def fisher_norm_sq(K, normalise=True):
 
 
 def sampled_fisher_norm_sq(X, dY, off, sample_rows):
-    """Squared Fisher norm of every sequence gradient as Algorithm 1 estimates it, from
-    `n_overlap_samples` token rows (`sample_rows`, drawn by the caller: the listing's `randperm`).
+    """Squared Fisher norm of every sequence gradient from sampled token positions (Sec. 2.2,
+    Eq. formal-F-norm with the "Efficient implementation" identities Eq. one and Eq. two).
 
-    a0 = act_in[samples], g0 = g_out[samples]; per sequence, with G_i = grad_out.T @ act_in,
-        F_norm = ||sum((g0 @ G_i) * a0, dim=1)|| / || ||g0_j|| * ||a0_j|| ||
-    i.e. the last display of "Efficient implementation" (Eq. one over Eq. two).  Returns F_norm^2, [B].
+    Sample j is the token gradient of row r_j = sample_rows[j] (drawn by the caller), the rank-one matrix
+    g_j = dY[r_j] X[r_j]^T.  For v = G_i the estimator is
+        F_i^2 = sum_j <G_i, g_j>^2 / sum_j ||g_j||^2,
+    with <G_i, g_j> = dY[r_j] . (G_i X[r_j])      (Eq. one: the overlap with a rank-one matrix)
+    and  ||g_j||^2  = ||dY[r_j]||^2 ||X[r_j]||^2  (Eq. two).
+    Every G_i is materialised.  Returns F^2, [B].
     """
     X, dY = _f64(X), _f64(dY)
     off = np.asarray(off, dtype=np.int64)
-    rows = np.asarray(sample_rows, dtype=np.int64)
-    a0 = X[rows]
-    g0 = dY[rows]
-    denom = np.linalg.norm(np.linalg.norm(g0, axis=1) * np.linalg.norm(a0, axis=1))
+    r = np.asarray(sample_rows, dtype=np.int64)
+    x_s, d_s = X[r], dY[r]
+    sample_norms_sq = np.sum(d_s * d_s, axis=1) * np.sum(x_s * x_s, axis=1)
+    total = np.sum(sample_norms_sq)
     B = off.shape[0] - 1
     F2 = np.empty(B, dtype=np.float64)
     for i in range(B):
-        seq = slice(int(off[i]), int(off[i + 1]))
-        seq_logprob_grad = dY[seq].T @ X[seq]
-        F_norm = np.linalg.norm(np.sum((g0 @ seq_logprob_grad) * a0, axis=1)) / denom
-        F2[i] = F_norm ** 2
+        lo, hi = int(off[i]), int(off[i + 1])
+        G_i = dY[lo:hi].T @ X[lo:hi]
+        overlaps = np.array([d_s[j] @ (G_i @ x_s[j]) for j in range(r.shape[0])])
+        F2[i] = np.sum(overlaps ** 2) / total
     return F2
 
 
