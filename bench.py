@@ -29,8 +29,9 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-# profiles/k_bf16_seq_grad_pair_gate_proj_32seq.md: (995.5 + 827.6) MB measured / 1711 MB algorithmic
-SEQ_GRAD_DRAM_OVER_ALGORITHMIC = 1.066
+# profiles/dram_traffic_llm_1p5b_block_full_size.md: 54.2 GB measured over the seven launches of the block at full
+# size / 51.5 GB algorithmic (inputs read once + stored gradients written once)
+SEQ_GRAD_DRAM_OVER_ALGORITHMIC = 1.052
 METRIC = "isopo_block_tokens_per_s"
 UNIT = "tokens/s"
 L2_BYTES = 126 * 1024 * 1024
@@ -441,15 +442,15 @@ def run_gpu(args):
     elif dom == "k_bf16_seq_grad":
         ms_total, n = prof[dom]
         achieved = flops_dw * args.steps / (ms_total * 1e-3) / 1e12
-        # DRAM bytes per launch: the ncu capture of this kernel on a smaller case (gate_proj, 32 sequences:
-        # 1.806 GB measured against 1.711 GB of inputs read once + gradients written once) scaled to the
-        # average launch of this run by its algorithmic bytes, to which the traffic is proportional.
+        # DRAM bytes per launch: ncu's dram__bytes_read + write of this kernel over the seven projections of the
+        # llm_1p5b block at full size (one-pass capture), as a ratio to the algorithmic bytes (inputs read once +
+        # gradients written once) and applied to this run's average launch.
         alg_bytes = sum(2.0 * T * (L["layer"].d_in + L["layer"].d_out) + 2.0 * B * L["layer"].d_in * L["layer"].d_out
                         for L in layers) / len(layers)
         traffic = SEQ_GRAD_DRAM_OVER_ALGORITHMIC * alg_bytes
         roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                    "traffic_unit": "bytes per launch (ncu dram__bytes_read+write on a smaller case, scaled)",
+                    "traffic_unit": "bytes per launch (ncu dram__bytes_read+write at full size on llm_1p5b: 1.052 x algorithmic)",
                     "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
                     "avg_launch_ms": ms_total / n, "launches": n}
     elif dom is not None:
