@@ -159,6 +159,27 @@ ISOPO_API isopo_status isopo_layer_gram_shared_x(const void* X, int n_proj, cons
                                                  size_t ws_bytes, int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_layer_gram_shared_x_stored: isopo_layer_gram on the MATERIALISE route for up to three
+ * projections that read the same input X (Alg. 2 reduce loop and NTK, per layer).  All projections'
+ * G_i = dY_i^(h)T X_i are formed by ONE launch of the per-sequence gradient GEMM: their tile rows are
+ * stacked into one grid, so X is staged once for all of them and narrow projections (the k/v shapes)
+ * no longer leave the machine half empty; K^(h) = G^(h) G^(h)T follows per projection.  bfloat16 only,
+ * B <= 256; results bit-identical to n_proj calls of isopo_layer_gram with ISOPO_PATH_MATERIALISE except for
+ * the order of the float atomic additions into K.
+ *
+ *   dY, d_out, K   HOST arrays of n_proj entries as for isopo_layer_gram_shared_x
+ *   ws, ws_bytes   HOST arrays: ws[h] is projection h's own workspace of at least
+ *                  isopo_workspace_bytes(dtype, T, d_in, d_out[h], B, ISOPO_PATH_MATERIALISE) bytes (1024-byte
+ *                  aligned, all distinct); it receives that projection's stored gradients and tag
+ * Follow it with isopo_weight_grad(X, dY[h], ..., ISOPO_PATH_MATERIALISE, ..., ws[h], ...) per projection.
+ */
+ISOPO_API isopo_status isopo_layer_gram_shared_x_stored(const void* X, int n_proj, const void* const* dY, const int* d_out,
+                                                        isopo_dtype dtype, int64_t T, int d_in,
+                                                        const int64_t* seq_offsets_host, int B, float* const* K,
+                                                        void* const* ws, const size_t* ws_bytes, int32_t* info,
+                                                        void* cuda_stream);
+
+/*
  * isopo_transform_advantages: advantages A -> coefficients c (dW = sum_i c_i G_i).
  *
  * With F_i^2 = sum_j K_ij^2 / sum_j K_jj (the Fisher norm of Eq. F-norm-basic evaluated with the B

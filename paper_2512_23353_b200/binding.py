@@ -28,6 +28,7 @@ INFO_STALE_WORKSPACE = 0x10000000
 EXPORTS = (
     "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",
     "isopo_layer_gram", "isopo_transform_advantages", "isopo_weight_grad", "isopo_layer_gram_shared_x",
+    "isopo_layer_gram_shared_x_stored",
     "isopo_profile_enable", "isopo_profile_collect", "isopo_kernel_name", "isopo_layer_gram_static",
     "isopo_sampled_workspace_bytes", "isopo_sampled_coefficients",
     "isopo_reg_ema_update", "isopo_transform_advantages_rel", "isopo_transform_advantages_batched",
@@ -67,6 +68,10 @@ def _load():
     lib.isopo_layer_gram_shared_x.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int,
                                               c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
                                               c.c_void_p]
+    lib.isopo_layer_gram_shared_x_stored.restype = c.c_int
+    lib.isopo_layer_gram_shared_x_stored.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_int64,
+                                                     c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p,
+                                                     c.c_void_p, c.c_void_p]
     lib.isopo_transform_advantages.restype = c.c_int
     lib.isopo_transform_advantages.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
                                                c.c_void_p, c.c_void_p, c.c_void_p]
@@ -194,6 +199,27 @@ def isopo_layer_gram_shared_x(X: torch.Tensor, dYs, seq_offsets, Ks, ws: torch.T
                                        X.shape[0], X.shape[1], off.ctypes.data, B, k_ptrs.ctypes.data, ws.data_ptr(),
                                        ws.numel(), info.data_ptr(), _stream())
     _check(st, "isopo_layer_gram_shared_x")
+
+
+def isopo_layer_gram_shared_x_stored(X: torch.Tensor, dYs, seq_offsets, Ks, wss, info: torch.Tensor) -> None:
+    """Stored-gradient-route K of up to three projections dYs[h] that share the input X: one launch forms all
+    their per-sequence gradients; wss[h] is projection h's own workspace (MATERIALISE size)."""
+    off = _offsets(seq_offsets)
+    B = off.shape[0] - 1
+    n = len(dYs)
+    assert len(Ks) == n and len(wss) == n and X.is_cuda and X.is_contiguous()
+    for dY, K, ws in zip(dYs, Ks, wss):
+        assert dY.is_cuda and dY.is_contiguous() and dY.dtype == X.dtype and dY.shape[0] == X.shape[0]
+        assert K.dtype == torch.float32 and K.is_contiguous() and K.numel() == B * B and ws.dtype == torch.uint8
+    dy_ptrs = np.array([d.data_ptr() for d in dYs], dtype=np.uint64)
+    k_ptrs = np.array([K.data_ptr() for K in Ks], dtype=np.uint64)
+    ws_ptrs = np.array([w.data_ptr() for w in wss], dtype=np.uint64)
+    ws_sizes = np.array([w.numel() for w in wss], dtype=np.uint64)
+    widths = np.array([d.shape[1] for d in dYs], dtype=np.int32)
+    st = lib.isopo_layer_gram_shared_x_stored(X.data_ptr(), n, dy_ptrs.ctypes.data, widths.ctypes.data, _dtype_code(X),
+                                              X.shape[0], X.shape[1], off.ctypes.data, B, k_ptrs.ctypes.data,
+                                              ws_ptrs.ctypes.data, ws_sizes.ctypes.data, info.data_ptr(), _stream())
+    _check(st, "isopo_layer_gram_shared_x_stored")
 
 
 def isopo_layer_gram_static(X: torch.Tensor, dY: torch.Tensor, seq_offsets, K: torch.Tensor,

@@ -278,6 +278,56 @@ isopo_status isopo_layer_gram_shared_x(const void* X, int n_proj, const void* co
   return bf16_gram_shared(X, dY, T, d_in, d_out, n_proj, tokseq, B, K, info, st);
 }
 
+isopo_status isopo_layer_gram_shared_x_stored(const void* X, int n_proj, const void* const* dY, const int* d_out,
+                                              isopo_dtype dtype, int64_t T, int d_in, const int64_t* seq_offsets_host, int B,
+                                              float* const* K, void* const* ws, const size_t* ws_bytes, int32_t* info,
+                                              void* cuda_stream) {
+  ApiRange nvtx_range("isopo_layer_gram_shared_x_stored");
+  if (!dY || !d_out || !K || !ws || !ws_bytes || !info || n_proj < 1 || n_proj > 3) return ISOPO_ERR_INVALID_ARG;
+  if (dtype != ISOPO_BF16 || B > 256) return ISOPO_ERR_UNSUPPORTED;
+  WsLayout L[3];
+  WsTag tag[3];
+  int64_t* off_dev[3];
+  int32_t* order[3];
+  WsTag* tag_dev[3];
+  void* G[3];
+  bool pairs_fit = true;
+  for (int h = 0; h < n_proj; ++h) {
+    if (!K[h]) return ISOPO_ERR_INVALID_ARG;
+    isopo_status s = check_layer_args(X, dY[h], dtype, T, d_in, d_out[h], seq_offsets_host, B, ISOPO_PATH_MATERIALISE, ws[h]);
+    if (s != ISOPO_OK) return s;
+    for (int g = 0; g < h; ++g)
+      if (ws[g] == ws[h]) return ISOPO_ERR_INVALID_ARG;  // every projection keeps its own gradients
+    L[h] = ws_layout(dtype, T, d_in, d_out[h], B, ISOPO_PATH_MATERIALISE);
+    if (ws_bytes[h] < L[h].total) return ISOPO_ERR_WORKSPACE;
+    char* w = (char*)ws[h];
+    tag[h] = make_ws_tag(dtype, T, d_in, d_out[h], B, seq_offsets_host);
+    off_dev[h] = (int64_t*)(w + L[h].off_offsets);
+    order[h] = (int32_t*)(w + L[h].off_order);
+    tag_dev[h] = (WsTag*)(w + L[h].off_tag);
+    G[h] = w + L[h].off_G;
+    pairs_fit = pairs_fit && (L[h].tiles_m % 2 == 0 || L[h].tiles_m >= 7);
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  isopo_status s = launch_prep_stored_multi(seq_offsets_host, B, n_proj, tag, off_dev, order, tag_dev, K, st);
+  if (s != ISOPO_OK) return s;
+  if (pairs_fit) {
+    s = bf16_seq_grad_pair_shared(X, n_proj, dY, d_out, T, d_in, off_dev[0], order[0], B, L, G, info, st);
+    if (s != ISOPO_OK) return s;
+  } else {  // a projection with an odd, small number of 128-row tiles would idle half of its pairs: one launch each
+    for (int h = 0; h < n_proj; ++h) {
+      s = bf16_seq_grad(X, dY[h], T, d_in, d_out[h], seq_offsets_host, off_dev[h], order[h], B, L[h], G[h], info, st);
+      if (s != ISOPO_OK) return s;
+    }
+  }
+  for (int h = 0; h < n_proj; ++h) {
+    float* kpart = deterministic_mode() ? (float*)((char*)ws[h] + L[h].off_kpart) : nullptr;
+    s = bf16_ntk(G[h], L[h], B, K[h], /*k_is_zero=*/true, kpart, info, st);
+    if (s != ISOPO_OK) return s;
+  }
+  return ISOPO_OK;
+}
+
 size_t isopo_sampled_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, int n_samples) {
   if (!sizes_ok(dtype, T, d_in, d_out, B) || n_samples < 1 || n_samples > ISOPO_MAX_SAMPLES) return 0;
   return sampled_layout(dtype, T, d_in, d_out, B, n_samples).total;

@@ -123,6 +123,8 @@ isopo_status launch_prep(const int64_t* off_host, int B, int64_t T, int64_t* off
 // bf16 materialised path (B <= 256) in one launch: offsets, the longest-first order, the workspace tag, K = 0
 isopo_status launch_prep_stored(const int64_t* off_host, int B, const WsTag& tag, int64_t* off_dev, int32_t* order_dev,
                                 WsTag* tag_dev, float* K, cudaStream_t st);
+isopo_status launch_prep_stored_multi(const int64_t* off_host, int B, int n_proj, const WsTag* tag, int64_t* const* off_dev,
+                                      int32_t* const* order_dev, WsTag* const* tag_dev, float* const* K, cudaStream_t st);
 isopo_status store_tag(const WsTag& tag, WsTag* tag_dev, cudaStream_t st);
 // offsets to the device and tokscale[t] = coeffs[sequence of token t] (float32 [T])
 isopo_status launch_tokscale(const int64_t* off_host, int B, int64_t T, int64_t* off_dev, const float* coeffs,
@@ -157,6 +159,10 @@ isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, i
 isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
                                 const int32_t* order_dev, int B, const WsLayout& L, void* G, int32_t* info,
                                 cudaStream_t st);
+// the same for up to three projections that read one X, in one launch (L, dY, d_out, G: one entry per projection)
+isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* const* dY, const int* d_out, int64_t T, int d_in,
+                                       const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout* L,
+                                       void* const* G, int32_t* info, cudaStream_t st);
 // k_is_zero: the caller has already cleared K on this stream.  kpart != NULL (deterministic mode): every CTA
 // stores its partial upper triangle there ([kNtkMaxPartials][B * B] floats) and a second kernel sums them in order.
 constexpr int kNtkMaxPartials = 160;

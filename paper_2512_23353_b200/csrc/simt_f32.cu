@@ -23,20 +23,25 @@ __global__ void k_store_offsets(OffsetArgs a, int base, int n, int64_t* __restri
 
 // Everything the bf16 stored-gradient kernels need before they start, in one launch (B <= 256):
 // CTA 0 leaves the offsets, the working order of the sequences and the workspace tag; all CTAs clear K.
+// With several projections sharing one launch (same offsets, one workspace each) every workspace gets its copy.
 struct StoredPrepArgs {
   int64_t off[257];
-  WsTag tag;
+  WsTag tag[3];
+  int64_t* off_dev[3];
+  int32_t* order_dev[3];
+  WsTag* tag_dev[3];
+  float* K[3];
   uint8_t order[256];
 };
-__global__ void __launch_bounds__(256) k_prep_stored(StoredPrepArgs a, int B, int64_t* __restrict__ off,
-                                                     int32_t* __restrict__ order, WsTag* __restrict__ tag,
-                                                     float* __restrict__ K) {
-  if (blockIdx.x == 0) {
-    for (int i = threadIdx.x; i <= B; i += blockDim.x) off[i] = a.off[i];
-    for (int i = threadIdx.x; i < B; i += blockDim.x) order[i] = a.order[i];
-    if (threadIdx.x < 8) tag->v[threadIdx.x] = a.tag.v[threadIdx.x];
+__global__ void __launch_bounds__(256) k_prep_stored(StoredPrepArgs a, int B, int n_proj) {
+  for (int h = 0; h < n_proj; ++h) {
+    if (blockIdx.x == 0) {
+      for (int i = threadIdx.x; i <= B; i += blockDim.x) a.off_dev[h][i] = a.off[i];
+      for (int i = threadIdx.x; i < B; i += blockDim.x) a.order_dev[h][i] = a.order[i];
+      if (threadIdx.x < 8) a.tag_dev[h]->v[threadIdx.x] = a.tag[h].v[threadIdx.x];
+    }
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < B * B; e += gridDim.x * blockDim.x) a.K[h][e] = 0.f;
   }
-  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < B * B; e += gridDim.x * blockDim.x) K[e] = 0.f;
 }
 __global__ void k_store_tag(WsTag t, WsTag* __restrict__ tag) {
   if (threadIdx.x < 8) tag->v[threadIdx.x] = t.v[threadIdx.x];
@@ -309,10 +314,18 @@ isopo_status launch_tokscale(const int64_t* off_host, int B, int64_t T, int64_t*
 
 isopo_status launch_prep_stored(const int64_t* off_host, int B, const WsTag& tag, int64_t* off_dev, int32_t* order_dev,
                                 WsTag* tag_dev, float* K, cudaStream_t st) {
-  if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  return launch_prep_stored_multi(off_host, B, 1, &tag, &off_dev, &order_dev, &tag_dev, &K, st);
+}
+
+isopo_status launch_prep_stored_multi(const int64_t* off_host, int B, int n_proj, const WsTag* tag, int64_t* const* off_dev,
+                                      int32_t* const* order_dev, WsTag* const* tag_dev, float* const* K, cudaStream_t st) {
+  if (B > 256 || n_proj < 1 || n_proj > 3) return ISOPO_ERR_UNSUPPORTED;
   StoredPrepArgs a;
   for (int i = 0; i <= B; ++i) a.off[i] = off_host[i];
-  a.tag = tag;
+  for (int h = 0; h < 3; ++h) {
+    const int hh = h < n_proj ? h : 0;
+    a.tag[h] = tag[hh]; a.off_dev[h] = off_dev[hh]; a.order_dev[h] = order_dev[hh]; a.tag_dev[h] = tag_dev[hh]; a.K[h] = K[hh];
+  }
   int idx[256];
   for (int i = 0; i < B; ++i) idx[i] = i;
   // longest first; equal lengths keep their order
@@ -320,7 +333,7 @@ isopo_status launch_prep_stored(const int64_t* off_host, int B, const WsTag& tag
   for (int i = 0; i < B; ++i) a.order[i] = (uint8_t)idx[i];
   {
     LaunchScope scope(kIdPrep, st);
-    k_prep_stored<<<std::max(1, (B * B + 2047) / 2048), 256, 0, st>>>(a, B, off_dev, order_dev, tag_dev, K);
+    k_prep_stored<<<std::max(1, (B * B + 2047) / 2048), 256, 0, st>>>(a, B, n_proj);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

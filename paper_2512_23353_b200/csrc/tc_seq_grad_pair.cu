@@ -17,6 +17,11 @@
 //   warps 2-5       epilogue: TMEM -> registers -> bf16 (round to nearest even) -> stored gradients
 //   warp 6          zeroes the dY rows past the end of a sequence in its last slab
 //
+// Several projections that read the same X (q/k/v, gate/up of a transformer block) can share one launch:
+// their pair-tile rows are stacked into one tile grid, the dY operand and the destination of a unit
+// come from the projection its row belongs to, and X is staged exactly as for one projection, so the
+// pairs running at one time share its tokens in L2 across projections as well.
+//
 // Barriers.  full[s] lives in CTA 0 and counts the bytes of both CTAs; tcgen05.commit releases
 // empty[s] and raises accfull[b] in BOTH CTAs; accempty[b] in CTA 0 counts the eight epilogue warps
 // of the pair.  In the last slab of a sequence whose length is not a multiple of 16 the dY copy of
@@ -51,16 +56,27 @@ constexpr int kPairN = 256;                          // columns of a pair tile (
 static_assert(kKB % 16 == 0 && kKB <= 256, "a stage is a whole number of 16-token MMA steps and one TMA box");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory");
 
+constexpr int kMaxProj = 3;  // projections sharing X in one launch
 struct PairParams {
   const int64_t* off;
   const int32_t* order;     // the k-th sequence to work on (longest first)
-  __nv_bfloat16* G;
-  int B, tiles_m, tiles_n;  // stored 128 x 256 tiles per gradient
-  int ptiles_m;             // pair tiles along d_out = ceil(tiles_m / 2)
+  __nv_bfloat16* G[kMaxProj];   // stored gradients of every projection
+  int tiles_m[kMaxProj];        // stored 128-row tiles of every projection
+  int ptm_first[kMaxProj + 1];  // first pair-tile row of every projection in the stacked grid
+  int n_proj;
+  int B, tiles_n;           // sequences; stored 256-column tiles per gradient (X is common)
+  int ptiles_m;             // pair-tile rows of the stacked grid = sum over projections of ceil(tiles_m / 2)
   int32_t* info;
   int group_m;              // pair-tile rows per group of the tile order
-  long long n_slots;        // 16-byte slots of the stored gradients (debug build: every store is checked against it)
+  long long n_slots[kMaxProj];  // 16-byte slots of each projection's stored gradients (debug build: every store is checked)
 };
+
+// projection that pair-tile row `ptm` of the stacked grid belongs to
+__device__ __forceinline__ int proj_of(const PairParams& p, int ptm) {
+  int h = 0;
+  while (h + 1 < p.n_proj && ptm >= p.ptm_first[h + 1]) ++h;
+  return h;
+}
 
 // The pair tiles of one sequence are visited in groups of `group_m` rows, row index fastest inside a
 // group: the ~74 pairs then work on about group_m row blocks of dY and 74 / group_m column blocks of X
@@ -92,7 +108,8 @@ __device__ __forceinline__ UnitShape unit_shape(int len) {
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapX, PairParams p) {
+k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_constant__ CUtensorMap mapY1,
+                     const __grid_constant__ CUtensorMap mapY2, const __grid_constant__ CUtensorMap mapX, PairParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
@@ -148,7 +165,9 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (elect_one()) {
-      prefetch_tensormap(&mapY);
+      prefetch_tensormap(&mapY0);
+      if (p.n_proj > 1) prefetch_tensormap(&mapY1);
+      if (p.n_proj > 2) prefetch_tensormap(&mapY2);
       prefetch_tensormap(&mapX);
       const uint32_t full_at_leader = map_to_cta(full_bar(0), 0);
       int stage = 0;
@@ -160,7 +179,9 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
         pair_tile(pt, p, ptm, tn);
         const int64_t t0 = s_first[k];
         const UnitShape us = unit_shape(s_len[k]);
-        const int ycol = (2 * ptm + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
+        const int h = proj_of(p, ptm);
+        const CUtensorMap* mapY = h == 0 ? &mapY0 : h == 1 ? &mapY1 : &mapY2;
+        const int ycol = (2 * (ptm - p.ptm_first[h]) + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
         for (int kb = 0; kb < us.nkb; ++kb) {
           if (!(ok = mbar_wait_pair(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kOperandBytes;
@@ -171,8 +192,8 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
           const uint32_t fb = full_at_leader + 8u * stage;
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
-            if (own_tail) tma_load_2d(a_dst + c * kChunkBytes, &mapY, ycol + c * 64, y, tail_bar(stage));
-            else tma_load_2d_pair(a_dst + c * kChunkBytes, &mapY, ycol + c * 64, y, fb);
+            if (own_tail) tma_load_2d(a_dst + c * kChunkBytes, mapY, ycol + c * 64, y, tail_bar(stage));
+            else tma_load_2d_pair(a_dst + c * kChunkBytes, mapY, ycol + c * 64, y, fb);
             tma_load_2d_pair(b_dst + c * kChunkBytes, &mapX, xcol + c * 64, y, fb);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -221,18 +242,19 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
     // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t accempty_at_leader = map_to_cta(accempty_bar(0), 0);
-    uint4* dst = reinterpret_cast<uint4*>(p.G);
     int acc = 0;
     uint32_t acc_phase = 0;
     for (long long u = pair_id; u < total_units; u += npairs) {
       const int i = s_seq[u / ptiles], pt = (int)(u % ptiles);
       int ptm, tn;
       pair_tile(pt, p, ptm, tn);
-      const int tm = 2 * ptm + (int)rank;
+      const int h = proj_of(p, ptm);
+      const int tm = 2 * (ptm - p.ptm_first[h]) + (int)rank;
       const int tile = tm * p.tiles_n + tn;
+      uint4* dst = reinterpret_cast<uint4*>(p.G[h]);
       if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
       tc_fence_after_sync();
-      if (tm < p.tiles_m) {  // an odd number of row tiles leaves the last pair's second half empty
+      if (tm < p.tiles_m[h]) {  // an odd number of row tiles leaves the last pair's second half empty
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
 #pragma unroll 2
         for (int jc = 0; jc < kPairN / 32; ++jc) {
@@ -247,7 +269,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
             o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
             o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
             const size_t slot = stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane);
-            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, p.n_slots, p.info, kIdSeqGrad)) dst[slot] = o;
+            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, p.n_slots[h], p.info, kIdSeqGrad)) dst[slot] = o;
           }
         }
       }
@@ -303,20 +325,36 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY, const __grid_cons
 isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
                                 const int32_t* order_dev, int B, const WsLayout& L, void* G, int32_t* info,
                                 cudaStream_t st) {
-  CUtensorMap mapY, mapX;
-  isopo_status s = make_map_2d_bf16(&mapY, dY, (uint64_t)T, (uint64_t)d_out, (uint64_t)d_out, 64, kKB);
-  if (s != ISOPO_OK) return s;
-  s = make_map_2d_bf16(&mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kKB);
+  const void* dYs[1] = {dY};
+  const int d_outs[1] = {d_out};
+  void* Gs[1] = {G};
+  return bf16_seq_grad_pair_shared(X, 1, dYs, d_outs, T, d_in, off_dev, order_dev, B, &L, Gs, info, st);
+}
+
+isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* const* dY, const int* d_out, int64_t T, int d_in,
+                                       const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout* L,
+                                       void* const* G, int32_t* info, cudaStream_t st) {
+  if (n_proj < 1 || n_proj > kMaxProj) return ISOPO_ERR_INVALID_ARG;
+  CUtensorMap mapY[kMaxProj], mapX;
+  PairParams p{};
+  p.off = off_dev; p.order = order_dev; p.B = B; p.tiles_n = L[0].tiles_n; p.n_proj = n_proj; p.info = info;
+  for (int h = 0; h < kMaxProj; ++h) {
+    const int hh = h < n_proj ? h : 0;  // unused slots repeat the first projection (never addressed)
+    isopo_status s = make_map_2d_bf16(&mapY[h], dY[hh], (uint64_t)T, (uint64_t)d_out[hh], (uint64_t)d_out[hh], 64, kKB);
+    if (s != ISOPO_OK) return s;
+    p.G[h] = (__nv_bfloat16*)G[hh];
+    p.tiles_m[h] = L[hh].tiles_m;
+    p.n_slots[h] = (long long)B * L[hh].n_pad / 8;
+    p.ptm_first[h] = h == 0 ? 0 : p.ptm_first[h - 1] + (h - 1 < n_proj ? (L[h - 1].tiles_m + 1) / 2 : 0);
+  }
+  p.ptm_first[kMaxProj] = p.ptm_first[kMaxProj - 1] + (kMaxProj - 1 < n_proj ? (L[kMaxProj - 1].tiles_m + 1) / 2 : 0);
+  p.ptiles_m = p.ptm_first[n_proj];
+  isopo_status s = make_map_2d_bf16(&mapX, X, (uint64_t)T, (uint64_t)d_in, (uint64_t)d_in, 64, kKB);
   if (s != ISOPO_OK) return s;
   int dev = 0, sms = 0;
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  PairParams p{};
-  p.off = off_dev; p.order = order_dev; p.G = (__nv_bfloat16*)G; p.B = B; p.tiles_m = L.tiles_m; p.tiles_n = L.tiles_n;
-  p.ptiles_m = (L.tiles_m + 1) / 2;
-  p.info = info;
-  p.n_slots = (long long)B * L.n_pad / 8;
   const long long units = (long long)B * p.ptiles_m * p.tiles_n;
   // Persistent pairs with a static share of the units each: launch only as many pairs as can be
   // resident at once (the hardware may place fewer 2-CTA clusters than there are SM pairs).
@@ -343,7 +381,7 @@ isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_
   p.group_m = std::max(1, std::min(g, p.ptiles_m));
   {
     LaunchScope scope(kIdSeqGrad, st);
-    k_bf16_seq_grad_pair<<<2 * npairs, kThreads, kSmemBytes, st>>>(mapY, mapX, p);
+    k_bf16_seq_grad_pair<<<2 * npairs, kThreads, kSmemBytes, st>>>(mapY[0], mapY[1], mapY[2], mapX, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
