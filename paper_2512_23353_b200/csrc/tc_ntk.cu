@@ -218,6 +218,10 @@ __global__ void k_mirror_upper(float* __restrict__ K, int B) {
   if (j < i) K[e] = K[(size_t)j * B + i];
 }
 
+#ifndef ISOPO_COMBINE_IN_FLIGHT
+#define ISOPO_COMBINE_IN_FLIGHT 16
+#endif
+constexpr int kCombineInFlight = ISOPO_COMBINE_IN_FLIGHT;  // 16-byte loads a thread has in flight
 // dW = beta dW + sum_i c_i G_i.  One thread per 16-byte slot of the piece-blocked store.
 __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long nchunks /* n_pad / 8 */,
                                                        int B, int tiles_n, int d_in, int d_out,
@@ -241,12 +245,12 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ 
     const uint4* src = G + stored_slot((size_t)piece, 0, B, l);
     const size_t chunks = 32;  // uint4 stride between successive sequences of one piece
     int i = 0;
-    for (; i + 8 <= B; i += 8) {
-      uint4 v[8];
+    for (; i + kCombineInFlight <= B; i += kCombineInFlight) {
+      uint4 v[kCombineInFlight];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(i + u) * chunks);
+      for (int u = 0; u < kCombineInFlight; ++u) v[u] = __ldcs(src + (size_t)(i + u) * chunks);
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < kCombineInFlight; ++u) {
         const float c = sc[i + u];
         const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
