@@ -71,11 +71,14 @@ struct PairParams {
   long long n_slots[kMaxProj];  // 16-byte slots of each projection's stored gradients (debug build: every store is checked)
 };
 
-// projection that pair-tile row `ptm` of the stacked grid belongs to
+// projection that pair-tile row `ptm` of the stacked grid belongs to (no indexing by a run-time value anywhere
+// below: that would move the parameter arrays to local memory)
 __device__ __forceinline__ int proj_of(const PairParams& p, int ptm) {
-  int h = 0;
-  while (h + 1 < p.n_proj && ptm >= p.ptm_first[h + 1]) ++h;
-  return h;
+  return (int)(p.n_proj > 1 && ptm >= p.ptm_first[1]) + (int)(p.n_proj > 2 && ptm >= p.ptm_first[2]);
+}
+template <typename T>
+__device__ __forceinline__ T pick(const T (&a)[kMaxProj], int h) {
+  return h == 0 ? a[0] : (h == 1 ? a[1] : a[2]);
 }
 
 // The pair tiles of one sequence are visited in groups of `group_m` rows, row index fastest inside a
@@ -181,7 +184,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
         const UnitShape us = unit_shape(s_len[k]);
         const int h = proj_of(p, ptm);
         const CUtensorMap* mapY = h == 0 ? &mapY0 : h == 1 ? &mapY1 : &mapY2;
-        const int ycol = (2 * (ptm - p.ptm_first[h]) + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
+        const int ycol = (2 * (ptm - (h == 0 ? 0 : (h == 1 ? p.ptm_first[1] : p.ptm_first[2]))) + (int)rank) * kHalf, xcol = tn * kPairN + (int)rank * kHalf;
         for (int kb = 0; kb < us.nkb; ++kb) {
           if (!(ok = mbar_wait_pair(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort, p.info, kIdSeqGrad))) break;
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kOperandBytes;
@@ -249,12 +252,12 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
       int ptm, tn;
       pair_tile(pt, p, ptm, tn);
       const int h = proj_of(p, ptm);
-      const int tm = 2 * (ptm - p.ptm_first[h]) + (int)rank;
+      const int tm = 2 * (ptm - (h == 0 ? 0 : (h == 1 ? p.ptm_first[1] : p.ptm_first[2]))) + (int)rank;
       const int tile = tm * p.tiles_n + tn;
-      uint4* dst = reinterpret_cast<uint4*>(p.G[h]);
+      uint4* dst = reinterpret_cast<uint4*>(pick(p.G, h));
       if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
       tc_fence_after_sync();
-      if (tm < p.tiles_m[h]) {  // an odd number of row tiles leaves the last pair's second half empty
+      if (tm < pick(p.tiles_m, h)) {  // an odd number of row tiles leaves the last pair's second half empty
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
 #pragma unroll 2
         for (int jc = 0; jc < kPairN / 32; ++jc) {
@@ -269,7 +272,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
             o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
             o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
             const size_t slot = stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane);
-            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, p.n_slots[h], p.info, kIdSeqGrad)) dst[slot] = o;
+            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, pick(p.n_slots, h), p.info, kIdSeqGrad)) dst[slot] = o;
           }
         }
       }
