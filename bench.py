@@ -279,6 +279,8 @@ def run_gpu(args):
     variant = b.VAR_INTERACTING if args.variant == "interacting" else b.VAR_NORMALISED
 
     sampled = args.route == "sampled"
+    if args.store_format == "e4m3_split":  # before any workspace is sized or written
+        b.isopo_set_store_format(b.STORE_E4M3_SPLIT)
     # Algorithm 1 draws its overlap samples with randperm: the bench draws them once, seeded, on the host
     sample_rows = np.random.default_rng(w.seed + 17).permutation(T)[: args.samples].astype(np.int64)
     # the stored route keeps every projection's workspace until the block's coefficients are known, so
@@ -640,6 +642,46 @@ def run_gpu(args):
             "clocks": s_clocks}}
         del s_ws
 
+    # ---- the stored route once more with the split e4m3 store (K pass on half the bytes), same inputs and workspaces ----
+    if not sampled and w.dtype == "bf16" and world == 1 and not args.skip_routes and args.store_format == "bf16":
+        b.isopo_set_store_format(b.STORE_E4M3_SPLIT)
+        try:
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            b.isopo_profile_collect()
+            n_s = max(1, min(args.steps, 10))
+            f_sampler = ClockSampler(local)
+            b.isopo_profile_enable(True)
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            f_sampler.start()
+            a.record()
+            for _ in range(n_s):
+                step()
+            c.record()
+            torch.cuda.synchronize()
+            f_clocks = f_sampler.stop()
+            b.isopo_profile_enable(False)
+            f_prof = b.isopo_profile_collect()
+            if int(info.item()) != 0:
+                raise SystemExit(f"device-side error with the split store: info={int(info.item()):#x}")
+            f_ms = a.elapsed_time(c) / n_s
+            from oracle import isopo_oracle as orc
+            f_parity = None if args.skip_parity else parity_check(
+                layers, off, A, [L["lam"] for L in layers], orc.INTERACTING if args.variant == "interacting" else orc.NORMALISED)
+            routes = routes or {}
+            routes["stored_e4m3_split"] = {
+                "what": "the stored route with isopo_set_store_format(ISOPO_STORE_E4M3_SPLIT): gradients kept as two e4m3 "
+                        "planes, K pass on the high plane, diagonal of K from float32 sums in the gradient GEMM; same "
+                        "inputs, workspaces and schedule, same run",
+                "ms_per_step": f_ms, "steps": n_s, "tokens_per_s": T / (f_ms * 1e-3),
+                "overhead_vs_plain_dw_gemm": f_ms / plain_ms,
+                "kernels": {k: {"ms_per_step": v[0] / n_s, "launches_per_step": v[1] / n_s} for k, v in f_prof.items()},
+                "parity": f_parity, "clocks": f_clocks}
+        finally:
+            b.isopo_set_store_format(b.STORE_BF16)
+
     # ---- the oracle on this machine's host cores, bounded sample ----
     cpu = None
     if world == 1 and not args.skip_cpu:
@@ -673,6 +715,7 @@ def run_gpu(args):
         "config": {"workload": args.workload, "B": B, "tokens": T,
                    "route": "sampled (Algorithm 1, %d token samples)" % len(sample_rows) if sampled else "stored gradients",
                    "variant": "normalised (Algorithm 1)" if sampled else args.variant,
+                   "store_format": args.store_format,
                    "layers": cfg_layers, "paths": cfg_paths,
                    "l2": ("L2 flushed between steps (256 MB fill, untimed); every step timed by its own events"
                           if flush else "inputs larger than L2 (no flush needed)"),
@@ -715,6 +758,8 @@ def main():
                     help="stored: K from materialised per-sequence gradients (both variants); sampled: Algorithm 1's "
                          "token-sampled Fisher norm + folded weight-gradient GEMM (non-interacting variant)")
     ap.add_argument("--samples", type=int, default=128, help="n_overlap_samples of the sampled route")
+    ap.add_argument("--store-format", default="bf16", choices=["bf16", "e4m3_split"],
+                    help="stored route: how the per-sequence gradients are kept (isopo_set_store_format)")
     ap.add_argument("--schedule", default="batched", choices=["batched", "single"],
                     help="stored route: batched = every projection keeps its workspace and one launch solves for all "
                          "their coefficients; single = one call per projection, one shared workspace")

@@ -396,6 +396,25 @@ ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, is
  * data-dependent index of the kernels is then range-checked before use, a violation skips the access
  * and sets *info = ISOPO_INFO_BOUNDS | kernel id.
  */
+/*
+ * Store format of the bf16 MATERIALISE route (the paper has no counterpart; SURVEY's "fp8 storage of G for the K
+ * pass").  ISOPO_STORE_BF16 (default): every G_i is kept as bf16.  ISOPO_STORE_E4M3_SPLIT: every element is kept as
+ * two e4m3 bytes, hi = round(s_i g) and lo = round(16 (s_i g - hi)), in two planes (the same 2 bytes per element; s_i
+ * a power of two per sequence, estimated from a sample of the sequence's token rows).  The K pass then reads only the
+ * hi plane - half the bytes, kind::f8f6f4 tensor-core instructions, about 0.6 x the time - and takes the diagonal of K
+ * from float32 sums of squares that the gradient GEMM forms from its accumulators (more exact than the bf16
+ * store's); the weight gradient reads both planes (8 significant bits, as bf16).  What it costs: the off-diagonal
+ * entries of K carry rounding noise of about 0.05 / sqrt(d_in d_out) of sqrt(K_ii K_jj), thirty times that of the
+ * bf16 store, which the interacting solve amplifies by cond(K + lambda I): meant for layers of a million weights and
+ * more and well-conditioned K; elements beyond 448 / s_i saturate.  Process-wide; set it before isopo_layer_gram and
+ * leave it unchanged until the layer's isopo_weight_grad (the workspace tag records the format, a mismatch is
+ * reported as ISOPO_INFO_STALE_WORKSPACE).  Layers that take the 1-CTA gradient kernel (an odd number, below 7, of
+ * 128-row tiles), ISOPO_F32 and deterministic mode keep the bf16 / float32 store.
+ */
+typedef enum { ISOPO_STORE_BF16 = 0, ISOPO_STORE_E4M3_SPLIT = 1 } isopo_store_format;
+ISOPO_API isopo_status isopo_set_store_format(isopo_store_format format);
+ISOPO_API isopo_store_format isopo_get_store_format(void);
+
 ISOPO_API void isopo_set_deterministic(int on);
 ISOPO_API int isopo_get_deterministic(void);
 ISOPO_API int isopo_debug_build(void);

@@ -34,6 +34,7 @@ EXPORTS = (
     "isopo_reg_ema_update", "isopo_transform_advantages_rel", "isopo_transform_advantages_batched",
     "isopo_spectral_workspace_bytes", "isopo_transform_spectral", "isopo_transform_spectral_batched",
     "isopo_selftest_bounded_wait", "isopo_set_deterministic", "isopo_get_deterministic", "isopo_debug_build",
+    "isopo_set_store_format", "isopo_get_store_format",
 )
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
@@ -105,6 +106,10 @@ def _load():
     lib.isopo_transform_advantages_rel.restype = c.c_int
     lib.isopo_transform_advantages_rel.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_float, c.c_void_p,
                                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.isopo_set_store_format.restype = c.c_int
+    lib.isopo_set_store_format.argtypes = [c.c_int]
+    lib.isopo_get_store_format.restype = c.c_int
+    lib.isopo_get_store_format.argtypes = []
     lib.isopo_set_deterministic.restype = None
     lib.isopo_set_deterministic.argtypes = [c.c_int]
     lib.isopo_get_deterministic.restype = c.c_int
@@ -387,6 +392,14 @@ def isopo_sampled_coefficients(X: torch.Tensor, dY: torch.Tensor, seq_offsets, s
                                         coeffs.data_ptr(), F2.data_ptr() if F2 is not None else None, ws.data_ptr(),
                                         ws.numel(), info.data_ptr(), _stream())
     _check(st, "isopo_sampled_coefficients")
+
+
+STORE_BF16, STORE_E4M3_SPLIT = 0, 1
+
+
+def isopo_set_store_format(fmt: int) -> None:
+    """Store format of the bf16 stored-gradient route: STORE_BF16 (default) or STORE_E4M3_SPLIT."""
+    _check(lib.isopo_set_store_format(int(fmt)), "isopo_set_store_format")
 
 
 def isopo_set_deterministic(on: bool) -> None:

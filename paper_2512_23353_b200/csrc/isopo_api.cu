@@ -30,6 +30,17 @@ void set_cuda_error(cudaError_t e, const char* where) {
 
 static bool g_deterministic = false;
 bool deterministic_mode() { return g_deterministic; }
+static isopo_store_format g_store_format = ISOPO_STORE_BF16;
+
+// The split store lives in the 2-CTA gradient GEMM and sums the diagonal of K with float atomics: layers that
+// take the 1-CTA kernel, and everything in deterministic mode, keep the bf16 store.
+bool use_split_store(const WsLayout& L, int B) {
+  return g_store_format == ISOPO_STORE_E4M3_SPLIT && !g_deterministic && B <= 256 && (L.tiles_m % 2 == 0 || L.tiles_m >= 7);
+}
+StoreFmt store_fmt(const WsLayout& L, int B, void* ws) {
+  float* aux = (float*)((char*)ws + L.off_aux);
+  return StoreFmt{use_split_store(L, B) ? 1 : 0, aux, aux + B};
+}
 
 // ---- measurement hooks ----
 struct ProfRecord { int id; cudaEvent_t a, b; };
@@ -71,6 +82,8 @@ WsLayout ws_layout(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, iso
   size_t p = 0;
   L.off_tag = p;
   p = align_up(p + sizeof(WsTag), 1024);
+  L.off_aux = p;
+  if (dtype == ISOPO_BF16 && resolved == ISOPO_PATH_MATERIALISE) p = align_up(p + 2 * sizeof(float) * (size_t)B, 1024);
   L.off_offsets = p;
   p = align_up(p + sizeof(int64_t) * (size_t)(B + 1), 1024);
   L.off_order = p;
@@ -110,6 +123,10 @@ WsTag make_ws_tag(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, cons
   WsTag t{};
   t.v[0] = 0x49534f504f5f4753ll;
   t.v[1] = (int64_t)dtype; t.v[2] = T; t.v[3] = d_in; t.v[4] = d_out; t.v[5] = B; t.v[6] = (int64_t)h;
+  if (dtype == ISOPO_BF16) {  // the format the stored gradients of this shape are kept in right now
+    const WsLayout L = ws_layout(dtype, T, d_in, d_out, B, ISOPO_PATH_MATERIALISE);
+    t.v[7] = use_split_store(L, B) ? 1 : 0;
+  }
   return t;
 }
 
@@ -160,6 +177,12 @@ const char* isopo_last_cuda_error(void) { return g_cuda_err; }
 void isopo_profile_enable(int on) { g_prof_on = on != 0; }
 
 void isopo_set_deterministic(int on) { g_deterministic = on != 0; }
+isopo_status isopo_set_store_format(isopo_store_format f) {
+  if (f != ISOPO_STORE_BF16 && f != ISOPO_STORE_E4M3_SPLIT) return ISOPO_ERR_INVALID_ARG;
+  g_store_format = f;
+  return ISOPO_OK;
+}
+isopo_store_format isopo_get_store_format(void) { return g_store_format; }
 int isopo_get_deterministic(void) { return g_deterministic ? 1 : 0; }
 int isopo_debug_build(void) {
 #ifdef ISOPO_DEBUG
@@ -236,9 +259,14 @@ isopo_status isopo_layer_gram(const void* X, const void* dY, isopo_dtype dtype, 
     s = launch_prep_stored(seq_offsets_host, B, make_ws_tag(dtype, T, d_in, d_out, B, seq_offsets_host), off_dev, order,
                            tag_dev, K, st);
     if (s != ISOPO_OK) return s;
-    s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, order, B, L, G, info, st);
+    const StoreFmt fmt = store_fmt(L, B, ws);
+    if (fmt.split) {
+      s = launch_seq_scales(X, dY, d_in, d_out, off_dev, B, (float*)fmt.scales, fmt.kdiag, st);
+      if (s != ISOPO_OK) return s;
+    }
+    s = bf16_seq_grad(X, dY, T, d_in, d_out, seq_offsets_host, off_dev, order, B, L, G, fmt, info, st);
     if (s != ISOPO_OK) return s;
-    return bf16_ntk(G, L, B, K, /*k_is_zero=*/true, deterministic_mode() ? (float*)(w + L.off_kpart) : nullptr, info, st);
+    return bf16_ntk(G, L, B, K, /*k_is_zero=*/true, deterministic_mode() ? (float*)(w + L.off_kpart) : nullptr, fmt, info, st);
   }
   s = launch_prep(seq_offsets_host, B, T, off_dev, tokseq, st);
   if (s != ISOPO_OK) return s;
@@ -291,6 +319,7 @@ isopo_status isopo_layer_gram_shared_x_stored(const void* X, int n_proj, const v
   int32_t* order[3];
   WsTag* tag_dev[3];
   void* G[3];
+  StoreFmt fmt[3];
   bool pairs_fit = true;
   for (int h = 0; h < n_proj; ++h) {
     if (!K[h]) return ISOPO_ERR_INVALID_ARG;
@@ -306,23 +335,29 @@ isopo_status isopo_layer_gram_shared_x_stored(const void* X, int n_proj, const v
     order[h] = (int32_t*)(w + L[h].off_order);
     tag_dev[h] = (WsTag*)(w + L[h].off_tag);
     G[h] = w + L[h].off_G;
+    fmt[h] = store_fmt(L[h], B, ws[h]);
     pairs_fit = pairs_fit && (L[h].tiles_m % 2 == 0 || L[h].tiles_m >= 7);
   }
   cudaStream_t st = (cudaStream_t)cuda_stream;
   isopo_status s = launch_prep_stored_multi(seq_offsets_host, B, n_proj, tag, off_dev, order, tag_dev, K, st);
   if (s != ISOPO_OK) return s;
+  for (int h = 0; h < n_proj; ++h)
+    if (fmt[h].split) {
+      s = launch_seq_scales(X, dY[h], d_in, d_out[h], off_dev[0], B, (float*)fmt[h].scales, fmt[h].kdiag, st);
+      if (s != ISOPO_OK) return s;
+    }
   if (pairs_fit) {
-    s = bf16_seq_grad_pair_shared(X, n_proj, dY, d_out, T, d_in, off_dev[0], order[0], B, L, G, info, st);
+    s = bf16_seq_grad_pair_shared(X, n_proj, dY, d_out, T, d_in, off_dev[0], order[0], B, L, G, fmt, info, st);
     if (s != ISOPO_OK) return s;
   } else {  // a projection with an odd, small number of 128-row tiles would idle half of its pairs: one launch each
     for (int h = 0; h < n_proj; ++h) {
-      s = bf16_seq_grad(X, dY[h], T, d_in, d_out[h], seq_offsets_host, off_dev[h], order[h], B, L[h], G[h], info, st);
+      s = bf16_seq_grad(X, dY[h], T, d_in, d_out[h], seq_offsets_host, off_dev[h], order[h], B, L[h], G[h], fmt[h], info, st);
       if (s != ISOPO_OK) return s;
     }
   }
   for (int h = 0; h < n_proj; ++h) {
     float* kpart = deterministic_mode() ? (float*)((char*)ws[h] + L[h].off_kpart) : nullptr;
-    s = bf16_ntk(G[h], L[h], B, K[h], /*k_is_zero=*/true, kpart, info, st);
+    s = bf16_ntk(G[h], L[h], B, K[h], /*k_is_zero=*/true, kpart, fmt[h], info, st);
     if (s != ISOPO_OK) return s;
   }
   return ISOPO_OK;
@@ -459,7 +494,7 @@ isopo_status isopo_weight_grad(const void* X, const void* dY, isopo_dtype dtype,
     const WsTag* tag_dev = (const WsTag*)(w + L.off_tag);
     if (dtype == ISOPO_F32)
       return f32_combine((const float*)(w + L.off_G), L.n_pad, B, coeffs, dW, beta, tag_dev, tag, info, st);
-    return bf16_combine(w + L.off_G, L, d_in, d_out, B, coeffs, dW, beta, tag_dev, tag, info, st);
+    return bf16_combine(w + L.off_G, L, d_in, d_out, B, coeffs, dW, beta, tag_dev, tag, store_fmt(L, B, ws), info, st);
   }
   // GEMM over all tokens: refresh the token -> sequence map so the call also works on its own.
   int64_t* off_dev = (int64_t*)(w + L.off_offsets);

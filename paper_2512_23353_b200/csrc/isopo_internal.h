@@ -82,8 +82,19 @@ struct WsTag {
 };
 WsTag make_ws_tag(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, const int64_t* off_host);
 
+// How the bf16 stored route keeps G_i.  Split (isopo_set_store_format(ISOPO_STORE_E4M3_SPLIT)): two e4m3 planes of
+// one byte per element each - `hi` = round(s_i G_i), `lo` = round(16 (s_i G_i - hi)) with a power-of-two scale s_i per
+// sequence - in the same piece order.  The K pass reads only `hi` (half the bytes, kind::f8f6f4 MMAs) and takes the
+// diagonal from `kdiag`, which the gradient GEMM sums in float32 from its accumulators; the combine reads both planes.
+struct StoreFmt {
+  int split;             // 0: bf16 (2 bytes per element), 1: e4m3 hi / lo planes
+  const float* scales;   // [B] s_i
+  float* kdiag;          // [B] sum of squares of G_i
+};
+
 struct WsLayout {
   size_t off_tag;      // WsTag (materialised path)
+  size_t off_aux;      // float scales[B] | float kdiag[B]  (bf16 materialised path, split store)
   size_t off_offsets;  // int64 [B+1]
   size_t off_order;    // int32 [B]       (bf16 materialised path: sequences, longest first)
   size_t off_tokseq;   // int32 [T]: token -> sequence; the bf16 weight-gradient GEMM keeps float32 per-token scales here
@@ -155,24 +166,31 @@ isopo_status f32_weight_grad(const float* X, const float* dY, int64_t T, int d_i
 // bf16 tcgen05 path
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
                            const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout& L, void* G,
-                           int32_t* info, cudaStream_t st);
+                           const StoreFmt& fmt, int32_t* info, cudaStream_t st);
 isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
-                                const int32_t* order_dev, int B, const WsLayout& L, void* G, int32_t* info,
-                                cudaStream_t st);
+                                const int32_t* order_dev, int B, const WsLayout& L, void* G, const StoreFmt& fmt,
+                                int32_t* info, cudaStream_t st);
+// whether a layer of this shape keeps its gradients in the split e4m3 format under the current settings
+bool use_split_store(const WsLayout& L, int B);
+StoreFmt store_fmt(const WsLayout& L, int B, void* ws);
+// s_i of every sequence from a sample of its token rows, kdiag = 0 (split store)
+isopo_status launch_seq_scales(const void* X, const void* dY, int d_in, int d_out, const int64_t* off_dev, int B, float* scales,
+                               float* kdiag, cudaStream_t st);
 // the same for up to three projections that read one X, in one launch (L, dY, d_out, G: one entry per projection)
 isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* const* dY, const int* d_out, int64_t T, int d_in,
                                        const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout* L,
-                                       void* const* G, int32_t* info, cudaStream_t st);
+                                       void* const* G, const StoreFmt* fmt, int32_t* info, cudaStream_t st);
 // k_is_zero: the caller has already cleared K on this stream.  kpart != NULL (deterministic mode): every CTA
 // stores its partial upper triangle there ([kNtkMaxPartials][B * B] floats) and a second kernel sums them in order.
 constexpr int kNtkMaxPartials = 160;
-isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, bool k_is_zero, float* kpart, int32_t* info,
-                      cudaStream_t st);
+isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, bool k_is_zero, float* kpart, const StoreFmt& fmt,
+                      int32_t* info, cudaStream_t st);
 bool deterministic_mode();
 // K[i][j] = K[j][i] for j < i (the K kernels fill the upper triangle)
-isopo_status mirror_upper(float* K, int B, cudaStream_t st);
+isopo_status mirror_upper(float* K, int B, cudaStream_t st, const float* kdiag = nullptr);
 isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
-                          float beta, const WsTag* tag_dev, const WsTag& tag, int32_t* info, cudaStream_t st);
+                          float beta, const WsTag* tag_dev, const WsTag& tag, const StoreFmt& fmt, int32_t* info,
+                          cudaStream_t st);
 isopo_status bf16_gram(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int32_t* tokseq, int B,
                        float* K, int32_t* info, cudaStream_t st);
 isopo_status bf16_gram_shared(const void* X, const void* const* dY, int64_t T, int d_in, const int* d_out, int n_heads,

@@ -5,6 +5,7 @@
 
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -49,6 +50,10 @@ isopo_status make_map_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows,
 // past B and pieces past the last read as zero.
 isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows,
                                   uint32_t box_pieces);
+// One e4m3 plane of the split store viewed as (x = byte inside a 256-byte piece row, y = sequence, z = piece): boxes of
+// 128 bytes x `box_rows` sequences x `box_pieces` pieces, 128-byte swizzle.
+isopo_status make_map_pieces_u8(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows,
+                                uint32_t box_pieces);
 
 // ---------------------------------------------------------------------------------------------
 // device: generic helpers
@@ -164,6 +169,15 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
       : "memory");
 }
+// The same with e4m3 A and B (kind::f8f6f4: 32 elements of the contraction per instruction, float32 accumulate).
+__device__ __forceinline__ void mma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         bool accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
 // Arrives on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -262,6 +276,11 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn, 
          | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// Instruction descriptor, kind::f8f6f4 with e4m3 A and B (format code 0), float32 D, both operands K-major.
+__host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N) {
+  return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
 // Shared-memory matrix descriptor for 128-byte-swizzled tiles (rows of 128 bytes, 8-row groups of
 // 1024 bytes, tile base 1024-byte aligned).
 //   K-major operand  (row = M/N index, 64 bf16 of K per row): sbo = bytes between 8-row groups.
@@ -276,6 +295,21 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // .x = lo (low 16 bits)
   return *reinterpret_cast<uint32_t*>(&v);
 }
+
+// two floats -> two e4m3 bytes (`a` in the low byte), round to nearest even, saturating at +-448
+__device__ __forceinline__ uint32_t pack_e4m3x2(float a, float b) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(b), "f"(a));
+  return r;
+}
+// two e4m3 bytes -> two halves / two floats (exact)
+__device__ __forceinline__ __half2 e4m3x2_to_half2(uint32_t v) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)v));
+  return *reinterpret_cast<__half2*>(&h2);
+}
+__device__ __forceinline__ float2 unpack_e4m3x2(uint32_t v) { return __half22float2(e4m3x2_to_half2(v)); }
+constexpr float kLoScale = 16.f;  // the `lo` plane of the split store holds 16 x the residual of the `hi` plane
 
 }  // namespace tc
 }  // namespace isopo

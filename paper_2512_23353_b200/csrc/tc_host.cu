@@ -72,5 +72,29 @@ isopo_status make_map_pieces_bf16(CUtensorMap* map, const void* base, uint64_t B
   return ISOPO_OK;
 }
 
+isopo_status make_map_pieces_u8(CUtensorMap* map, const void* base, uint64_t B, uint64_t pieces, uint32_t box_rows,
+                                uint32_t box_pieces) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) {
+    set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
+    return ISOPO_ERR_CUDA;
+  }
+  if (box_rows == 0 || box_rows > 256 || box_pieces == 0 || box_pieces > 256 || ((uintptr_t)base & 15) || B == 0 ||
+      pieces == 0)
+    return ISOPO_ERR_INVALID_ARG;
+  cuuint64_t dims[3] = {256, B, pieces};
+  cuuint64_t strides[2] = {256, B * 256};
+  cuuint32_t box[3] = {128, box_rows, box_pieces};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (e4m3 plane)");
+    return ISOPO_ERR_CUDA;
+  }
+  return ISOPO_OK;
+}
+
 }  // namespace tc
 }  // namespace isopo

@@ -36,6 +36,7 @@ constexpr uint32_t kTmemCols = 512;
 
 struct NtkParams {
   float* kpart;   // deterministic mode: [CTA][B * B] partial sums, plain stores; NULL: float atomics into K
+  const float* scales;  // split store: s_i per sequence (the `hi` plane holds s_i G_i); the diagonal is not written here
   float* K;
   int B;
   long long nkb;  // boxes in the contraction dimension: ceil(pieces / ppb) * 4
@@ -44,6 +45,9 @@ struct NtkParams {
   int ppb;        // pieces per box = 256 / box_rows
 };
 
+// kE4m3: the operand is the `hi` plane of the split store: 128 one-byte elements per 128-byte box row (two boxes
+// per piece instead of four), kind::f8f6f4 MMAs of 32 elements each - the same number of MMAs per byte, half the bytes.
+template <bool kE4m3>
 __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant__ CUtensorMap mapG, NtkParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -87,14 +91,17 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
         for (long long kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.info, kIdNtk)) break;
           mbar_arrive_expect_tx(full_bar(stage), stage_tx);
-          tma_load_3d(smem_base + stage * kStageBytes, &mapG, (int)(kb & 3) * kKB, 0, (int)(kb >> 2) * p.ppb, full_bar(stage));
+          if (kE4m3)
+            tma_load_3d(smem_base + stage * kStageBytes, &mapG, (int)(kb & 1) * 128, 0, (int)(kb >> 1) * p.ppb, full_bar(stage));
+          else
+            tma_load_3d(smem_base + stage * kStageBytes, &mapG, (int)(kb & 3) * kKB, 0, (int)(kb >> 2) * p.ppb, full_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     } else if (warp == 1) {
       if (elect_one()) {  // elected, not "lane 0": lets the compiler keep the MMA operands in uniform registers
-        const uint32_t idesc1 = make_idesc_bf16(128, n1, false, false);
-        const uint32_t idesc2 = make_idesc_bf16(128, n2, false, false);
+        const uint32_t idesc1 = kE4m3 ? make_idesc_e4m3(128, n1) : make_idesc_bf16(128, n1, false, false);
+        const uint32_t idesc2 = kE4m3 ? make_idesc_e4m3(128, n2) : make_idesc_bf16(128, n2, false, false);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -107,8 +114,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
             const bool accum = (kb > kb0) || k16 > 0;
             const uint64_t d0 = make_sdesc_sw128(base + k16 * 32, 16, 1024);
             const uint64_t d1 = make_sdesc_sw128(base + 128 * 128 + k16 * 32, 16, 1024);
-            mma_bf16(tmem_base, d0, d0, idesc1, accum);
-            mma_bf16(tmem_base + 256, d1, d1, idesc2, accum);
+            if (kE4m3) {
+              mma_e4m3(tmem_base, d0, d0, idesc1, accum);
+              mma_e4m3(tmem_base + 256, d1, d1, idesc2, accum);
+            } else {
+              mma_bf16(tmem_base, d0, d0, idesc1, accum);
+              mma_bf16(tmem_base + 256, d1, d1, idesc2, accum);
+            }
           }
           mma_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -123,8 +135,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
       auto add_to_k = [&](size_t idx, float v) {
         if (mine) mine[idx] = v; else atomicAdd(&p.K[idx], v);
       };
-      // `ok` is false only after a wait ran out; every thread still reaches the named barrier below
+      // `ok` is false only after a wait ran out; every thread still reaches the named barriers below
       const bool ok = mbar_wait(accfull_bar, 0, abort_flag, p.info, kIdNtk);
+      // split store: the accumulators hold s_i s_j <G_i, G_j>; 1 / s_i of every sequence goes to shared memory (the ring
+      // is idle by now), and the diagonal is left to the gradient GEMM's float32 sums
+      float* inv_s = reinterpret_cast<float*>(smem + 128 * 1024);
+      if (kE4m3) {
+        for (int i = r; i < 256; i += 128) inv_s[i] = i < p.B ? 1.f / __ldg(p.scales + i) : 0.f;
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+      }
+      auto unscale = [&](int row, int col, float v) { return kE4m3 ? v * inv_s[row] * inv_s[col] : v; };
       {
         tc_fence_after_sync();
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
@@ -138,8 +158,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const int c = c0 + e;
-                if (c >= r && c < p.B && ISOPO_IN_RANGE((long long)r * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
-                  add_to_k((size_t)r * p.B + c, __uint_as_float(v[e]));
+                if (c >= r + (kE4m3 ? 1 : 0) && c < p.B &&
+                    ISOPO_IN_RANGE((long long)r * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
+                  add_to_k((size_t)r * p.B + c, unscale(r, c, __uint_as_float(v[e])));
               }
             }
           }
@@ -153,8 +174,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const int c = 128 + c0 + e;
-                if (c >= rr && c < p.B && ISOPO_IN_RANGE((long long)rr * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
-                  add_to_k((size_t)rr * p.B + c, __uint_as_float(v[e]));
+                if (c >= rr + (kE4m3 ? 1 : 0) && c < p.B &&
+                    ISOPO_IN_RANGE((long long)rr * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
+                  add_to_k((size_t)rr * p.B + c, unscale(rr, c, __uint_as_float(v[e])));
               }
             }
           }
@@ -182,11 +204,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
           if (ok) {
             for (int idx = r; idx < (ncol << lr); idx += 128) {
               const int sq = idx & (rows - 1), c = idx >> lr;
-              if (c < sq || sq >= p.B) continue;  // upper triangle of the sequences that exist
+              if (c < sq + (kE4m3 ? 1 : 0) || sq >= p.B) continue;  // upper triangle of the sequences that exist
               float sum = 0.f;
               for (int h = 0; h < ngroups; ++h) sum += red[(((h << lr) + c) << lr) + sq];
               if (ISOPO_IN_RANGE((long long)sq * p.B + c, (long long)p.B * p.B, p.info, kIdNtk))
-                add_to_k((size_t)sq * p.B + c, sum);
+                add_to_k((size_t)sq * p.B + c, unscale(sq, c, sum));
             }
           }
         }
@@ -211,26 +233,31 @@ __global__ void k_ntk_reduce(const float* __restrict__ kpart, int n_ctas, int B,
   K[e] = s;
 }
 
-__global__ void k_mirror_upper(float* __restrict__ K, int B) {
+// kdiag != NULL (split store): the diagonal comes from the gradient GEMM's float32 sums of squares
+__global__ void k_mirror_upper(float* __restrict__ K, int B, const float* __restrict__ kdiag) {
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= B * B) return;
   const int i = e / B, j = e % B;
   if (j < i) K[e] = K[(size_t)j * B + i];
+  else if (j == i && kdiag) K[e] = kdiag[i];
 }
 
 #ifndef ISOPO_COMBINE_IN_FLIGHT
 #define ISOPO_COMBINE_IN_FLIGHT 16
 #endif
 constexpr int kCombineInFlight = ISOPO_COMBINE_IN_FLIGHT;  // 16-byte loads a thread has in flight
-// dW = beta dW + sum_i c_i G_i.  One thread per 16-byte slot of the piece-blocked store.
-__global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long nchunks /* n_pad / 8 */,
+// dW = beta dW + sum_i c_i G_i.  One thread per slot (8 elements of every G_i) of the piece-blocked store.
+// kSplit: the slot is 8 bytes in each of the two e4m3 planes, G_i = (hi + lo / 16) / s_i.
+template <bool kSplit>
+__global__ void __launch_bounds__(256) k_bf16_combine(const void* __restrict__ Gv, long long nchunks /* n_pad / 8 */,
                                                        int B, int tiles_n, int d_in, int d_out,
-                                                       const float* __restrict__ coeffs, float* __restrict__ dW,
-                                                       float beta, const WsTag* __restrict__ tag_dev, WsTag tag,
+                                                       const float* __restrict__ coeffs, const float* __restrict__ scales,
+                                                       float* __restrict__ dW, float beta,
+                                                       const WsTag* __restrict__ tag_dev, WsTag tag,
                                                        int32_t* __restrict__ info) {
   if (!ws_tag_matches(tag_dev, tag, info)) return;  // another layer's or microbatch's gradients: touch nothing
   __shared__ float sc[256];
-  for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = coeffs[i];
+  for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = kSplit ? coeffs[i] / scales[i] : coeffs[i];
   __syncthreads();
   for (long long pos = blockIdx.x * (long long)blockDim.x + threadIdx.x; pos < nchunks;
        pos += (long long)gridDim.x * blockDim.x) {
@@ -242,32 +269,59 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ 
     if (!ISOPO_IN_RANGE((long long)stored_slot((size_t)piece, B - 1, B, l), nchunks * B, info, kIdCombine)) continue;
     if (!ISOPO_IN_RANGE((long long)m * d_in + n + 7, (long long)d_out * d_in, info, kIdCombine)) continue;
     float acc[8] = {};
-    const uint4* src = G + stored_slot((size_t)piece, 0, B, l);
-    const size_t chunks = 32;  // uint4 stride between successive sequences of one piece
-    int i = 0;
-    for (; i + kCombineInFlight <= B; i += kCombineInFlight) {
-      uint4 v[kCombineInFlight];
+    const size_t first = stored_slot((size_t)piece, 0, B, l);
+    const size_t stride = 32;  // slots between successive sequences of one piece
+    if (kSplit) {
+      const uint2* hi = static_cast<const uint2*>(Gv) + first;
+      const uint2* lo = hi + (size_t)nchunks * B;
+      constexpr int kN = kCombineInFlight / 2;
+      int i = 0;
+      auto add = [&](const uint2& hv, const uint2& lv, float c) {
+        const uint32_t hw[4] = {hv.x & 0xffffu, hv.x >> 16, hv.y & 0xffffu, hv.y >> 16};
+        const uint32_t lw[4] = {lv.x & 0xffffu, lv.x >> 16, lv.y & 0xffffu, lv.y >> 16};
 #pragma unroll
-      for (int u = 0; u < kCombineInFlight; ++u) v[u] = __ldcs(src + (size_t)(i + u) * chunks);
+        for (int h = 0; h < 4; ++h) {
+          // hi + lo / 16 in half precision is exact (4 + 4 significant bits, at most 9 binades apart)
+          const float2 g = __half22float2(__hfma2(e4m3x2_to_half2(lw[h]), __float2half2_rn(1.f / kLoScale), e4m3x2_to_half2(hw[h])));
+          acc[2 * h] = fmaf(c, g.x, acc[2 * h]);
+          acc[2 * h + 1] = fmaf(c, g.y, acc[2 * h + 1]);
+        }
+      };
+      for (; i + kN <= B; i += kN) {
+        uint2 hv[kN], lv[kN];
 #pragma unroll
-      for (int u = 0; u < kCombineInFlight; ++u) {
-        const float c = sc[i + u];
-        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        for (int u = 0; u < kN; ++u) { hv[u] = __ldcs(hi + (size_t)(i + u) * stride); lv[u] = __ldcs(lo + (size_t)(i + u) * stride); }
+#pragma unroll
+        for (int u = 0; u < kN; ++u) add(hv[u], lv[u], sc[i + u]);
+      }
+      for (; i < B; ++i) add(__ldcs(hi + (size_t)i * stride), __ldcs(lo + (size_t)i * stride), sc[i]);
+    } else {
+      const uint4* src = static_cast<const uint4*>(Gv) + first;
+      int i = 0;
+      for (; i + kCombineInFlight <= B; i += kCombineInFlight) {
+        uint4 v[kCombineInFlight];
+#pragma unroll
+        for (int u = 0; u < kCombineInFlight; ++u) v[u] = __ldcs(src + (size_t)(i + u) * stride);
+#pragma unroll
+        for (int u = 0; u < kCombineInFlight; ++u) {
+          const float c = sc[i + u];
+          const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {
+            acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
+            acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
+          }
+        }
+      }
+      for (; i < B; ++i) {
+        const uint4 v = __ldcs(src + (size_t)i * stride);
+        const float c = sc[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
           acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
           acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
         }
-      }
-    }
-    for (; i < B; ++i) {
-      const uint4 v = __ldcs(src + (size_t)i * chunks);
-      const float c = sc[i];
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int h = 0; h < 4; ++h) {
-        acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
-        acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
       }
     }
     float4* out = reinterpret_cast<float4*>(dW + (size_t)m * d_in + n);
@@ -284,28 +338,33 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ 
 
 }  // namespace
 
-isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, bool k_is_zero, float* kpart, int32_t* info,
-                      cudaStream_t st) {
+isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, bool k_is_zero, float* kpart, const StoreFmt& fmt,
+                      int32_t* info, cudaStream_t st) {
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
+  if (fmt.split && kpart) return ISOPO_ERR_INVALID_ARG;  // the split store's diagonal is summed with float atomics
   CUtensorMap mapG;
   const uint32_t rows = B > 128 ? 256 : B > 64 ? 128 : B > 32 ? 64 : 32, ppb = 256 / rows;
   const long long pieces = L.n_pad / kPieceElems;
-  isopo_status s = make_map_pieces_bf16(&mapG, G, (uint64_t)B, (uint64_t)pieces, rows, ppb);
+  isopo_status s = fmt.split ? make_map_pieces_u8(&mapG, G, (uint64_t)B, (uint64_t)pieces, rows, ppb)
+                             : make_map_pieces_bf16(&mapG, G, (uint64_t)B, (uint64_t)pieces, rows, ppb);
   if (s != ISOPO_OK) return s;
   int dev = 0, sms = 0;
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_ntk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  auto kernel = fmt.split ? k_bf16_ntk<true> : k_bf16_ntk<false>;
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   if (!k_is_zero && !kpart) ISOPO_CUDA_TRY(cudaMemsetAsync(K, 0, sizeof(float) * (size_t)B * B, st));
-  NtkParams p{kpart, K, B, (pieces + ppb - 1) / ppb * 4, info, (int)rows, (int)ppb};
+  // boxes along the contraction: four per piece group of bf16 (64 elements a row), two of e4m3 (128 elements a row)
+  NtkParams p{kpart, fmt.split ? fmt.scales : nullptr, K, B, (pieces + ppb - 1) / ppb * (fmt.split ? 2 : 4), info, (int)rows,
+              (int)ppb};
   int grid = (int)std::max<long long>(1, std::min<long long>(sms, p.nkb / 8));
   if (kpart) grid = std::min(grid, kNtkMaxPartials);
   {
     LaunchScope scope(kIdNtk, st);
-    k_bf16_ntk<<<grid, kThreads, kSmemBytes, st>>>(mapG, p);
+    kernel<<<grid, kThreads, kSmemBytes, st>>>(mapG, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
-  if (!kpart) return mirror_upper(K, B, st);
+  if (!kpart) return mirror_upper(K, B, st, fmt.split ? fmt.kdiag : nullptr);
   // CTAs whose slab of the contraction is empty wrote nothing: sum only those that had work
   const long long per = (p.nkb + grid - 1) / grid;
   const int n_active = (int)((p.nkb + per - 1) / per);
@@ -317,17 +376,18 @@ isopo_status bf16_ntk(const void* G, const WsLayout& L, int B, float* K, bool k_
   return ISOPO_OK;
 }
 
-isopo_status mirror_upper(float* K, int B, cudaStream_t st) {
+isopo_status mirror_upper(float* K, int B, cudaStream_t st, const float* kdiag) {
   {
     LaunchScope scope(kIdMirror, st);
-    k_mirror_upper<<<(B * B + 255) / 256, 256, 0, st>>>(K, B);
+    k_mirror_upper<<<(B * B + 255) / 256, 256, 0, st>>>(K, B, kdiag);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
 }
 
 isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out, int B, const float* coeffs, float* dW,
-                          float beta, const WsTag* tag_dev, const WsTag& tag, int32_t* info, cudaStream_t st) {
+                          float beta, const WsTag* tag_dev, const WsTag& tag, const StoreFmt& fmt, int32_t* info,
+                          cudaStream_t st) {
   if (B > 256) return ISOPO_ERR_UNSUPPORTED;
   const long long chunks = L.n_pad / 8;
   int dev = 0, sms = 0;
@@ -336,7 +396,12 @@ isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out,
   const int grid = (int)std::min<long long>((chunks + 255) / 256, (long long)sms * 8);
   {
     LaunchScope scope(kIdCombine, st);
-    k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta, tag_dev, tag, info);
+    if (fmt.split)
+      k_bf16_combine<true><<<grid, 256, 0, st>>>(G, chunks, B, L.tiles_n, d_in, d_out, coeffs, fmt.scales, dW, beta, tag_dev,
+                                                 tag, info);
+    else
+      k_bf16_combine<false><<<grid, 256, 0, st>>>(G, chunks, B, L.tiles_n, d_in, d_out, coeffs, nullptr, dW, beta, tag_dev,
+                                                  tag, info);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

@@ -337,12 +337,13 @@ static isopo_status sm_count(int* sms) {
 
 isopo_status bf16_seq_grad(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_host,
                            const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout& L, void* G,
-                           int32_t* info, cudaStream_t st) {
+                           const StoreFmt& fmt, int32_t* info, cudaStream_t st) {
   (void)off_host;
   // 2-CTA tiles (256 rows of G per pair) when they waste little: an odd number of 128-row tiles
   // leaves half of the last pair idle.
   if (L.tiles_m % 2 == 0 || L.tiles_m >= 7)
-    return bf16_seq_grad_pair(X, dY, T, d_in, d_out, off_dev, order_dev, B, L, G, info, st);
+    return bf16_seq_grad_pair(X, dY, T, d_in, d_out, off_dev, order_dev, B, L, G, fmt, info, st);
+  if (fmt.split) return ISOPO_ERR_INVALID_ARG;  // the split store exists in the 2-CTA kernel only (use_split_store)
   CUtensorMap mapY, mapX;
   isopo_status s = make_maps(&mapY, &mapX, X, dY, T, d_in, d_out);
   if (s != ISOPO_OK) return s;

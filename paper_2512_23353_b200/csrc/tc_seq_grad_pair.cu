@@ -68,7 +68,10 @@ struct PairParams {
   int ptiles_m;             // pair-tile rows of the stacked grid = sum over projections of ceil(tiles_m / 2)
   int32_t* info;
   int group_m;              // pair-tile rows per group of the tile order
-  long long n_slots[kMaxProj];  // 16-byte slots of each projection's stored gradients (debug build: every store is checked)
+  long long n_slots[kMaxProj];  // slots (8 elements each) of each projection's stored gradients
+  // split e4m3 store (see StoreFmt; kernel instantiation kSplit): G[h] is then the `hi` plane, the `lo` plane follows it
+  const float* scales[kMaxProj];
+  float* kdiag[kMaxProj];
 };
 
 // projection that pair-tile row `ptm` of the stacked grid belongs to (no indexing by a run-time value anywhere
@@ -110,6 +113,7 @@ __device__ __forceinline__ UnitShape unit_shape(int len) {
   return s;
 }
 
+template <bool kSplit>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_constant__ CUtensorMap mapY1,
                      const __grid_constant__ CUtensorMap mapY2, const __grid_constant__ CUtensorMap mapX, PairParams p) {
@@ -257,7 +261,42 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
       uint4* dst = reinterpret_cast<uint4*>(pick(p.G, h));
       if (!mbar_wait_pair(accfull_bar(acc), acc_phase, abort_flag, peer_abort, p.info, kIdSeqGrad)) break;
       tc_fence_after_sync();
-      if (tm < pick(p.tiles_m, h)) {  // an odd number of row tiles leaves the last pair's second half empty
+      if (kSplit && tm < pick(p.tiles_m, h)) {
+        // split store: hi = e4m3(s_i g), lo = e4m3(16 (s_i g - hi)), 8 bytes per lane and plane; the sum of g^2 goes to kdiag
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
+        const long long n_slots = pick(p.n_slots, h);
+        uint2* hi_plane = reinterpret_cast<uint2*>(pick(p.G, h));
+        uint2* lo_plane = hi_plane + n_slots;
+        const float s_i = __ldg(pick(p.scales, h) + i);
+        float ksum = 0.f;
+#pragma unroll 2
+        for (int jc = 0; jc < kPairN / 32; ++jc) {
+          uint32_t r[32];
+          tmem_ld32(taddr + jc * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t hw[4], lw[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float g0 = __uint_as_float(r[v * 8 + 2 * e]), g1 = __uint_as_float(r[v * 8 + 2 * e + 1]);
+              ksum = fmaf(g0, g0, fmaf(g1, g1, ksum));
+              const float v0 = g0 * s_i, v1 = g1 * s_i;
+              hw[e] = pack_e4m3x2(v0, v1);
+              const float2 hf = unpack_e4m3x2(hw[e]);
+              lw[e] = pack_e4m3x2((v0 - hf.x) * kLoScale, (v1 - hf.y) * kLoScale);
+            }
+            const size_t slot = stored_slot(stored_piece(tile, jc * 4 + v, q), i, p.B, lane);
+            if (ISOPO_IN_RANGE(i < 0 || i >= p.B ? -1 : (long long)slot, n_slots, p.info, kIdSeqGrad)) {
+              hi_plane[slot] = make_uint2(hw[0] | (hw[1] << 16), hw[2] | (hw[3] << 16));
+              lo_plane[slot] = make_uint2(lw[0] | (lw[1] << 16), lw[2] | (lw[3] << 16));
+            }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ksum += __shfl_xor_sync(0xffffffffu, ksum, o);
+        if (lane == 0 && ISOPO_IN_RANGE(i, p.B, p.info, kIdSeqGrad)) atomicAdd(pick(p.kdiag, h) + i, ksum);
+      } else if (!kSplit && tm < pick(p.tiles_m, h)) {  // an odd number of row tiles leaves the last pair's second half empty
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
 #pragma unroll 2
         for (int jc = 0; jc < kPairN / 32; ++jc) {
@@ -323,21 +362,80 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
   if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
 }
 
+// Split store: a power-of-two scale per sequence that brings the typical element of G_i to about 2, where e4m3 has
+// its 3 mantissa bits with 2^8 of headroom and 2^7 below (sum_t dY_t x_t^T over L independent tokens has
+// elements of size sqrt(L) rms(dY) rms(x); fully correlated tokens give sqrt(L) times more, still in range).
+// The rms values come from up to 16 evenly spaced token rows of the sequence (16-byte loads: d_in and d_out are
+// multiples of 8).  Also clears kdiag.
+__device__ __forceinline__ float sum_sq8(const uint4& v) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  float s = 0.f;
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    const float a = __uint_as_float(w[h] << 16), b = __uint_as_float(w[h] & 0xffff0000u);
+    s = fmaf(a, a, fmaf(b, b, s));
+  }
+  return s;
+}
+__global__ void __launch_bounds__(512) k_seq_scales(const uint4* __restrict__ X, const uint4* __restrict__ dY, int d_in8,
+                                                    int d_out8, const int64_t* __restrict__ off,
+                                                    float* __restrict__ scales, float* __restrict__ kdiag) {
+  const int i = blockIdx.x;
+  const int64_t t0 = off[i], len = off[i + 1] - t0;
+  const int n = (int)min((int64_t)16, len);
+  float sx = 0.f, sy = 0.f;
+  for (int e = threadIdx.x; e < n * d_in8; e += blockDim.x) {
+    const int k = e / d_in8, c = e - k * d_in8;
+    sx += sum_sq8(__ldg(X + (t0 + (len * k) / n) * d_in8 + c));
+  }
+  for (int e = threadIdx.x; e < n * d_out8; e += blockDim.x) {
+    const int k = e / d_out8, c = e - k * d_out8;
+    sy += sum_sq8(__ldg(dY + (t0 + (len * k) / n) * d_out8 + c));
+  }
+  __shared__ float red[2][16];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { sx += __shfl_xor_sync(0xffffffffu, sx, o); sy += __shfl_xor_sync(0xffffffffu, sy, o); }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = sx; red[1][threadIdx.x >> 5] = sy; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    sx = sy = 0.f;
+    for (int w = 0; w < 16; ++w) { sx += red[0][w]; sy += red[1][w]; }
+    const float typical = sqrtf((float)len * (sx / ((float)n * 8.f * d_in8)) * (sy / ((float)n * 8.f * d_out8)));
+    // 2^k nearest to 2 / typical; inputs that are all zero (or not finite) keep the scale one
+    float s = 1.f;
+    if (typical > 0.f && typical < 3.0e38f) s = exp2f(rintf(log2f(2.f / typical)));
+    scales[i] = fminf(fmaxf(s, 1.0e-30f), 1.0e30f);
+    kdiag[i] = 0.f;
+  }
+}
+
 }  // namespace
 
+isopo_status launch_seq_scales(const void* X, const void* dY, int d_in, int d_out, const int64_t* off_dev, int B, float* scales,
+                               float* kdiag, cudaStream_t st) {
+  {
+    LaunchScope scope(kIdPrep, st);
+    k_seq_scales<<<B, 512, 0, st>>>((const uint4*)X, (const uint4*)dY, d_in / 8, d_out / 8, off_dev, scales, kdiag);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
 isopo_status bf16_seq_grad_pair(const void* X, const void* dY, int64_t T, int d_in, int d_out, const int64_t* off_dev,
-                                const int32_t* order_dev, int B, const WsLayout& L, void* G, int32_t* info,
-                                cudaStream_t st) {
+                                const int32_t* order_dev, int B, const WsLayout& L, void* G, const StoreFmt& fmt,
+                                int32_t* info, cudaStream_t st) {
   const void* dYs[1] = {dY};
   const int d_outs[1] = {d_out};
   void* Gs[1] = {G};
-  return bf16_seq_grad_pair_shared(X, 1, dYs, d_outs, T, d_in, off_dev, order_dev, B, &L, Gs, info, st);
+  return bf16_seq_grad_pair_shared(X, 1, dYs, d_outs, T, d_in, off_dev, order_dev, B, &L, Gs, &fmt, info, st);
 }
 
 isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* const* dY, const int* d_out, int64_t T, int d_in,
                                        const int64_t* off_dev, const int32_t* order_dev, int B, const WsLayout* L,
-                                       void* const* G, int32_t* info, cudaStream_t st) {
+                                       void* const* G, const StoreFmt* fmt, int32_t* info, cudaStream_t st) {
   if (n_proj < 1 || n_proj > kMaxProj) return ISOPO_ERR_INVALID_ARG;
+  for (int h = 1; h < n_proj; ++h)
+    if (fmt[h].split != fmt[0].split) return ISOPO_ERR_INVALID_ARG;  // one store format per launch
   CUtensorMap mapY[kMaxProj], mapX;
   PairParams p{};
   p.off = off_dev; p.order = order_dev; p.B = B; p.tiles_n = L[0].tiles_n; p.n_proj = n_proj; p.info = info;
@@ -348,6 +446,8 @@ isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* co
     p.G[h] = (__nv_bfloat16*)G[hh];
     p.tiles_m[h] = L[hh].tiles_m;
     p.n_slots[h] = (long long)B * L[hh].n_pad / 8;
+    p.scales[h] = fmt[hh].scales;
+    p.kdiag[h] = fmt[hh].kdiag;
     p.ptm_first[h] = h == 0 ? 0 : p.ptm_first[h - 1] + (h - 1 < n_proj ? (L[h - 1].tiles_m + 1) / 2 : 0);
   }
   p.ptm_first[kMaxProj] = p.ptm_first[kMaxProj - 1] + (kMaxProj - 1 < n_proj ? (L[kMaxProj - 1].tiles_m + 1) / 2 : 0);
@@ -357,12 +457,14 @@ isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* co
   int dev = 0, sms = 0;
   ISOPO_CUDA_TRY(cudaGetDevice(&dev));
   ISOPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_bf16_seq_grad_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  auto kernel = fmt[0].split ? k_bf16_seq_grad_pair<true> : k_bf16_seq_grad_pair<false>;
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   const long long units = (long long)B * p.ptiles_m * p.tiles_n;
   // Persistent pairs with a static share of the units each: launch only as many pairs as can be
   // resident at once (the hardware may place fewer 2-CTA clusters than there are SM pairs).
-  static int resident_pairs[64] = {};
+  static int resident[2][64] = {};
   if (dev < 0 || dev >= 64) return ISOPO_ERR_UNSUPPORTED;
+  int* resident_pairs = resident[fmt[0].split ? 1 : 0];
   if (resident_pairs[dev] == 0) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (unsigned)(sms / 2));
@@ -374,7 +476,7 @@ isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* co
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    ISOPO_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, k_bf16_seq_grad_pair, &cfg));
+    ISOPO_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kernel, &cfg));
     if (n < 1) return ISOPO_ERR_UNSUPPORTED;
     resident_pairs[dev] = std::min(n, sms / 2);
   }
@@ -384,7 +486,7 @@ isopo_status bf16_seq_grad_pair_shared(const void* X, int n_proj, const void* co
   p.group_m = std::max(1, std::min(g, p.ptiles_m));
   {
     LaunchScope scope(kIdSeqGrad, st);
-    k_bf16_seq_grad_pair<<<2 * npairs, kThreads, kSmemBytes, st>>>(mapY[0], mapY[1], mapY[2], mapX, p);
+    kernel<<<2 * npairs, kThreads, kSmemBytes, st>>>(mapY[0], mapY[1], mapY[2], mapX, p);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

@@ -28,6 +28,7 @@ def test_edge_shape_parity_on_the_range_checking_build():
     r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu",
                         "tests/test_parity_bf16.py", "tests/test_parity_f32.py", "tests/test_weight_grad_fold_gpu.py",
                         "tests/test_sampled_gpu.py", "tests/test_gram_shared_gpu.py", "tests/test_workspace_tag_gpu.py",
+                        "tests/test_shared_x_stored_gpu.py", "tests/test_split_store_gpu.py",
                         "-k", "not small_llm_config"],
                        cwd=ROOT, env=env, capture_output=True, text=True)
     tail = "\n".join(r.stdout.splitlines()[-15:])

@@ -1,0 +1,125 @@
+"""GPU parity of the bf16 stored-gradient route with the split e4m3 store (isopo_set_store_format): every G_i kept as
+two e4m3 planes, the K pass on the high plane alone (Alg. 2 "make neural tangent kernel" at half the bytes), the
+diagonal of K from float32 sums inside the gradient GEMM, the weight gradient (Alg. 2 last line) from both planes.
+Checked against the fp64 oracle: K within the 2e-2 of bf16 inputs overall, its diagonal far tighter, its off-diagonal
+entries on the Cauchy-Schwarz scale within the format's noise model, dW and the coefficients within 2e-2."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import isopo_oracle as orc
+from paper_2512_23353_b200 import workloads as wl
+from tests._util import rel_fro, report, to_f64
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+@pytest.fixture()
+def b():
+    from paper_2512_23353_b200 import binding
+    binding.isopo_set_store_format(binding.STORE_E4M3_SPLIT)
+    yield binding
+    binding.isopo_set_store_format(binding.STORE_BF16)
+
+
+def _inputs(Ls, d_in, d_out, seed, dy_scale=0.1, correlated=False):
+    rng = np.random.default_rng(seed)
+    off = np.concatenate([[0], np.cumsum(Ls)]).astype(np.int64)
+    w = wl.Workload("t", "bf16", len(Ls), "uniform", 1, 1, 4, "half", seed=seed)
+    X, dY = wl.layer_inputs_host(w, wl.LayerShape("l", d_in, d_out), int(off[-1]), correlated)
+    dY = dY * np.float32(dy_scale / 0.1)
+    A = rng.standard_normal(len(Ls)).astype(np.float32)
+    to = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)  # noqa: E731
+    return to(X), to(dY), off, torch.from_numpy(A).cuda()
+
+
+CASES = [
+    # (lengths, d_in, d_out, dY scale, correlated): every layer has an even number of 128-row tiles (2-CTA kernel)
+    ([1, 15, 16, 17, 63, 64, 65, 127, 129, 200], 256, 256, 0.1, False),     # ragged tails, B <= 32 box shape
+    ([700, 300, 1100], 1536, 256, 0.1, False),                              # 1.5B-class kv shape
+    (list(range(20, 90)), 320, 1000, 0.1, True),                            # B = 70, ragged widths, correlated tokens
+    (list(range(10, 150)), 264, 256, 0.1, False),                           # B = 140: two row blocks of K
+    ([40] * 256, 512, 256, 0.1, False),                                     # B = 256
+    ([300, 200, 250, 100], 256, 512, 1e-4, False),                          # tiny gradients: the scale brings them into range
+    ([300, 200, 250, 100], 256, 512, 3e3, True),                            # huge, correlated gradients
+]
+
+
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_split_store_matches_oracle(b, case):
+    Ls, d_in, d_out, dy_scale, correlated = CASES[case]
+    X, dY, off, A = _inputs(Ls, d_in, d_out, 6000 + case, dy_scale, correlated)
+    B, N = len(Ls), d_in * d_out
+    G = orc.sequence_gradients(to_f64(X), to_f64(dY), off)
+    K_o = orc.ntk(G)
+    lam = 1e-1 * float(np.mean(np.diag(K_o)))        # the mode is meant for well-conditioned K
+    res = b.isopo_layer(X, dY, off, A, b.VAR_INTERACTING, lam, b.PATH_MATERIALISE)
+    assert res.info == 0
+    K = res.K.cpu().numpy().astype(np.float64)
+    assert np.array_equal(K, K.T)
+    d, d_o = np.diag(K), np.diag(K_o)
+    scale = np.sqrt(np.outer(d_o, d_o))
+    off_err = np.abs(K - K_o) / scale
+    np.fill_diagonal(off_err, 0.0)
+    c_o = orc.transform_advantages(K_o, to_f64(A), orc.INTERACTING, lam)
+    errs = dict(K=rel_fro(K, K_o), K_diag=float(np.max(np.abs(d - d_o) / d_o)), K_offdiag_cs=float(off_err.max()),
+                noise_model=0.05 / np.sqrt(N), c=rel_fro(res.coeffs.cpu().numpy(), c_o),
+                dW=rel_fro(res.dW.cpu().numpy(), orc.weight_gradient(G, c_o)),
+                cond=float(np.linalg.cond(K_o + lam * np.eye(B))))
+    report(f"split store case {case} ({d_in}->{d_out}, B={B})", **errs)
+    assert errs["K"] <= TOL and errs["c"] <= TOL and errs["dW"] <= TOL, errs
+    assert errs["K_diag"] <= 1e-4, errs                     # float32 sums of squares of the accumulators
+    assert errs["K_offdiag_cs"] <= 8 * errs["noise_model"], errs   # worst entry of up to 256^2 against the rms model
+
+
+def test_split_store_full_size_projection(b):
+    """q_proj of the 1.5B-class block at full size (256 sequences, 334k tokens): K on a sample of sequences, a block of dW."""
+    w = wl.WORKLOADS["llm_1p5b"]
+    layer = next(l for l in w.layers if l.name == "q_proj")
+    off, A_host = wl.microbatch(w)
+    T, B = int(off[-1]), len(A_host)
+    X, dY = wl.layer_inputs_device(w, layer, T)
+    A = torch.from_numpy(A_host).cuda()
+    ws = b.alloc_workspace(b.BF16, T, layer.d_in, layer.d_out, B, b.PATH_MATERIALISE)
+    K = torch.empty(B, B, device="cuda")
+    c = torch.empty(B, device="cuda")
+    dW = torch.empty(layer.d_out, layer.d_in, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.isopo_layer_gram(X, dY, off, K, ws, info, b.PATH_MATERIALISE)
+    lam = 1e-3 * float(torch.diagonal(K).mean().item())
+    b.isopo_transform_advantages(K, A, b.VAR_INTERACTING, lam, c, info)
+    b.isopo_weight_grad(X, dY, c, off, dW, ws, info, b.PATH_MATERIALISE, 0.0)
+    torch.cuda.synchronize()
+    assert int(info.item()) == 0
+    L = np.diff(off)
+    pick = sorted(np.argsort(L)[:8].tolist())
+    rows = torch.cat([torch.arange(int(off[i]), int(off[i + 1])) for i in pick]).cuda()
+    off_s = np.concatenate([[0], np.cumsum([L[i] for i in pick])]).astype(np.int64)
+    K_s = orc.ntk(orc.sequence_gradients(to_f64(X[rows]), to_f64(dY[rows]), off_s))
+    K_gpu = K.cpu().numpy()[np.ix_(pick, pick)]
+    rng = np.random.default_rng(3)
+    m_idx = torch.from_numpy(np.sort(rng.choice(layer.d_out, size=32, replace=False))).cuda()
+    n_idx = torch.from_numpy(np.sort(rng.choice(layer.d_in, size=64, replace=False))).cuda()
+    G_blk = orc.sequence_gradients(to_f64(X[:, n_idx]), to_f64(dY[:, m_idx]), off)
+    errs = dict(K=rel_fro(K_gpu, K_s), K_diag=float(np.max(np.abs(np.diag(K_gpu) - np.diag(K_s)) / np.diag(K_s))),
+                dW=rel_fro(dW[m_idx][:, n_idx].cpu().numpy(), orc.weight_gradient(G_blk, to_f64(c))),
+                c_from_K=rel_fro(c.cpu().numpy(), orc.transform_advantages(to_f64(K), to_f64(A), orc.INTERACTING, lam)))
+    report("split store, llm_1p5b/q_proj at full size", **errs)
+    assert errs["K"] <= TOL and errs["K_diag"] <= 1e-4 and errs["dW"] <= TOL and errs["c_from_K"] <= 1e-4, errs
+
+
+def test_format_is_part_of_the_workspace_tag(b):
+    X, dY, off, A = _inputs([70, 130, 64], 256, 256, 61)
+    ws = b.alloc_workspace(b.BF16, int(off[-1]), 256, 256, 3, b.PATH_MATERIALISE)
+    K = torch.empty(3, 3, device="cuda")
+    info = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.isopo_layer_gram(X, dY, off, K, ws, info, b.PATH_MATERIALISE)          # split store
+    b.isopo_set_store_format(b.STORE_BF16)
+    dW = torch.full((256, 256), 7.0, device="cuda")
+    b.isopo_weight_grad(X, dY, A, off, dW, ws, info, b.PATH_MATERIALISE, 0.0)  # would read the planes as bf16
+    torch.cuda.synchronize()
+    assert int(info.item()) == b.INFO_STALE_WORKSPACE and bool((dW == 7.0).all())
+    with pytest.raises(b.IsopoError):
+        b.isopo_set_store_format(7)
