@@ -397,8 +397,8 @@ ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, is
  * and sets *info = ISOPO_INFO_BOUNDS | kernel id.
  */
 /*
- * Store format of the bf16 MATERIALISE route (the paper has no counterpart; SURVEY's "fp8 storage of G for the K
- * pass").  ISOPO_STORE_BF16 (default): every G_i is kept as bf16.  ISOPO_STORE_E4M3_SPLIT: every element is kept as
+ * Store format of the bf16 MATERIALISE route (the paper has no counterpart: an 8-bit storage of G for the K
+ * pass).  ISOPO_STORE_BF16 (default): every G_i is kept as bf16.  ISOPO_STORE_E4M3_SPLIT: every element is kept as
  * two e4m3 bytes, hi = round(s_i g) and lo = round(16 (s_i g - hi)), in two planes (the same 2 bytes per element; s_i
  * a power of two per sequence, estimated from a sample of the sequence's token rows).  The K pass then reads only the
  * hi plane - half the bytes, kind::f8f6f4 tensor-core instructions, about 0.6 x the time - and takes the diagonal of K
