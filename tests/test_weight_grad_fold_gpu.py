@@ -53,6 +53,7 @@ CASES = [
     ([513, 2047, 191, 1025], 264, 1000),                # 8 row tiles (the last one ragged), ragged columns
     ([4096], 256, 256),                                 # one sequence: every chunk is a slice of it
     ([150] * 40, 896, 896),                             # square, several chunks of several sequences
+    ([1, 1, 2, 15, 16, 17, 3000, 1, 63, 64, 65, 2000, 1, 1, 1, 640], 320, 256),   # runs of one-token segments between long ones
 ]
 
 
