@@ -30,7 +30,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 # profiles/dram_traffic_llm_1p5b_block_full_size.md: 80.3 GB measured over the seven launches of the block at full
-# size (median of four one-pass captures: 54.2, 80.3, 80.6, 86.4 GB) / 51.5 GB algorithmic (inputs read once +
+# size (median of five one-pass captures on five boxes: 54.2, 56.0, 80.2, 80.6, 86.4 GB) / 51.5 GB algorithmic (inputs read once +
 # stored gradients written once)
 SEQ_GRAD_DRAM_OVER_ALGORITHMIC = 1.56
 METRIC = "isopo_block_tokens_per_s"
@@ -453,7 +453,7 @@ def run_gpu(args):
         traffic = SEQ_GRAD_DRAM_OVER_ALGORITHMIC * alg_bytes
         roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                    "traffic_unit": "bytes per launch (ncu dram__bytes_read+write at full size on llm_1p5b, median of four boxes: 1.56 x algorithmic)",
+                    "traffic_unit": "bytes per launch (ncu dram__bytes_read+write at full size on llm_1p5b, median of five boxes: 1.56 x algorithmic)",
                     "peak_source": f"{peaks['source']} sustained bf16 (burst {peaks['bf16_tflops']})",
                     "avg_launch_ms": ms_total / n, "launches": n}
     elif dom is not None:
