@@ -102,6 +102,43 @@ def test_argument_validation_happens_on_the_host(binding):
     assert wg == b.ERR_INVALID_ARG                                     # beta must be 0 or 1
 
 
+def test_new_entry_points_validate_on_the_host(binding):
+    """The entry points added around the three calls reject bad arguments before any CUDA call, and the
+    process-wide switches change what they say they change (workspace size, nothing else)."""
+    b = binding
+    off = np.array([0, 3, 5], dtype=np.int64)
+    fake = 1 << 20
+    ptrs = np.array([fake, fake + (1 << 16), fake + (1 << 17)], dtype=np.uint64)
+    widths = np.array([8, 8, 8], dtype=np.int32)
+    sizes = np.array([1 << 30] * 3, dtype=np.uint64)
+    stored = lambda **kw: b.lib.isopo_layer_gram_shared_x_stored(  # noqa: E731
+        fake, kw.get("n", 2), ptrs.ctypes.data, widths.ctypes.data, kw.get("dtype", b.BF16), 5, 8, off.ctypes.data,
+        kw.get("B", 2), ptrs.ctypes.data, kw.get("ws", ptrs).ctypes.data, kw.get("sizes", sizes).ctypes.data, fake, None)
+    assert stored(n=0) == b.ERR_INVALID_ARG and stored(n=4) == b.ERR_INVALID_ARG
+    assert stored(dtype=b.F32) == b.ERR_UNSUPPORTED
+    assert stored(ws=np.array([fake, fake, fake], dtype=np.uint64)) == b.ERR_INVALID_ARG      # one workspace twice
+    assert stored(sizes=np.array([16, 16, 16], dtype=np.uint64)) == b.ERR_WORKSPACE
+    assert b.lib.isopo_selftest_bounded_wait(0, fake, fake, None) == b.ERR_INVALID_ARG
+    assert b.lib.isopo_selftest_bounded_wait(1000, None, fake, None) == b.ERR_INVALID_ARG
+    assert b.lib.isopo_set_store_format(5) == b.ERR_INVALID_ARG
+    assert b.lib.isopo_get_store_format() == b.STORE_BF16
+    base = b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_MATERIALISE)
+    b.isopo_set_store_format(b.STORE_E4M3_SPLIT)                      # the same two bytes per element
+    try:
+        assert b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_MATERIALISE) == base
+    finally:
+        b.isopo_set_store_format(b.STORE_BF16)
+    b.isopo_set_deterministic(True)                                   # per-CTA partial sums of K live in the workspace
+    try:
+        assert b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_MATERIALISE) >= base + 160 * 16 * 16 * 4
+        assert b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_GRAM) == \
+            b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_GRAM)
+    finally:
+        b.isopo_set_deterministic(False)
+    assert b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_MATERIALISE) == base
+    assert not b.isopo_debug_build()
+
+
 def test_binding_has_no_fallback():
     src = open(os.path.join(ROOT, "paper_2512_23353_b200", "binding.py")).read()
     assert "oracle" not in src.replace("CPU oracle", "")
