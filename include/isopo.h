@@ -89,6 +89,7 @@ typedef enum {
 
 #define ISOPO_INFO_TIMEOUT 0x40000000
 #define ISOPO_INFO_NO_CONVERGENCE 0x20000000 /* isopo_transform_spectral: sweeps ran out; low bits = sweeps done */
+#define ISOPO_INFO_SATURATED 0x04000000 /* split e4m3 store: an element of some s_i G_i exceeded the format's range (448) and was clamped */
 #define ISOPO_INFO_BOUNDS 0x08000000 /* debug build only (isopo_debug_build): kernel `id` computed an index outside its buffer; the access was skipped */
 #define ISOPO_INFO_STALE_WORKSPACE 0x10000000 /* isopo_weight_grad(MATERIALISE): the workspace holds another layer's or microbatch's gradients */
 
@@ -406,7 +407,8 @@ ISOPO_API isopo_status isopo_layer_gram_static(const void* X, const void* dY, is
  * store's); the weight gradient reads both planes (8 significant bits, as bf16).  What it costs: the off-diagonal
  * entries of K carry rounding noise of about 0.05 / sqrt(d_in d_out) of sqrt(K_ii K_jj), thirty times that of the
  * bf16 store, which the interacting solve amplifies by cond(K + lambda I): meant for layers of a million weights and
- * more and well-conditioned K; elements beyond 448 / s_i saturate.  Process-wide; set it before isopo_layer_gram and
+ * more and well-conditioned K; elements beyond 448 / s_i are clamped and reported (*info = ISOPO_INFO_SATURATED |
+ * kernel id: inputs with outlier channels hundreds of times the typical size need the bf16 store).  Process-wide; set it before isopo_layer_gram and
  * leave it unchanged until the layer's isopo_weight_grad (the workspace tag records the format, a mismatch is
  * reported as ISOPO_INFO_STALE_WORKSPACE).  Layers that take the 1-CTA gradient kernel (an odd number, below 7, of
  * 128-row tiles), ISOPO_F32 and deterministic mode keep the bf16 / float32 store.

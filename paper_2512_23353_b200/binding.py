@@ -24,6 +24,7 @@ PATH_AUTO, PATH_GRAM, PATH_MATERIALISE = 0, 1, 2
  VAR_NORMALISED_RAW) = range(7)
 INFO_TIMEOUT = 0x40000000
 INFO_STALE_WORKSPACE = 0x10000000
+INFO_SATURATED = 0x04000000
 
 EXPORTS = (
     "isopo_status_string", "isopo_last_cuda_error", "isopo_choose_path", "isopo_workspace_bytes",

@@ -268,7 +268,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
         uint2* hi_plane = reinterpret_cast<uint2*>(pick(p.G, h));
         uint2* lo_plane = hi_plane + n_slots;
         const float s_i = __ldg(pick(p.scales, h) + i);
-        float ksum = 0.f;
+        float ksum = 0.f, vmax = 0.f;
 #pragma unroll 2
         for (int jc = 0; jc < kPairN / 32; ++jc) {
           uint32_t r[32];
@@ -282,6 +282,7 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
               const float g0 = __uint_as_float(r[v * 8 + 2 * e]), g1 = __uint_as_float(r[v * 8 + 2 * e + 1]);
               ksum = fmaf(g0, g0, fmaf(g1, g1, ksum));
               const float v0 = g0 * s_i, v1 = g1 * s_i;
+              vmax = fmaxf(vmax, fmaxf(fabsf(v0), fabsf(v1)));
               hw[e] = pack_e4m3x2(v0, v1);
               const float2 hf = unpack_e4m3x2(hw[e]);
               lw[e] = pack_e4m3x2((v0 - hf.x) * kLoScale, (v1 - hf.y) * kLoScale);
@@ -296,6 +297,8 @@ k_bf16_seq_grad_pair(const __grid_constant__ CUtensorMap mapY0, const __grid_con
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ksum += __shfl_xor_sync(0xffffffffu, ksum, o);
         if (lane == 0 && ISOPO_IN_RANGE(i, p.B, p.info, kIdSeqGrad)) atomicAdd(pick(p.kdiag, h) + i, ksum);
+        // an element beyond e4m3's largest value was clamped: K and dW are off by more than rounding, say so
+        if (__any_sync(0xffffffffu, vmax > 448.f) && lane == 0) atomicCAS(p.info, 0, ISOPO_INFO_SATURATED | kIdSeqGrad);
       } else if (!kSplit && tm < pick(p.tiles_m, h)) {  // an odd number of row tiles leaves the last pair's second half empty
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kPairN;
 #pragma unroll 2

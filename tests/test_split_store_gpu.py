@@ -110,6 +110,22 @@ def test_split_store_full_size_projection(b):
     assert errs["K"] <= TOL and errs["K_diag"] <= 1e-4 and errs["dW"] <= TOL and errs["c_from_K"] <= 1e-4, errs
 
 
+def test_out_of_range_elements_are_reported(b):
+    """One token whose activations are ten thousand times the typical size, in a row that the scale estimate (the rms
+    of 16 evenly spaced rows per sequence) does not see: its products leave e4m3's range, are clamped, and the call
+    says so in *info instead of returning a quietly wrong K.  The same inputs on the bf16 store are fine."""
+    X, dY, off, A = _inputs([300, 200, 250, 100], 256, 512, 71)
+    X[7, :] *= 1.0e4
+    res = b.isopo_layer(X, dY, off, A, b.VAR_NORMALISED, 0.0, b.PATH_MATERIALISE)
+    probe = [k for k in range(b.NUM_KERNELS) if b.lib.isopo_kernel_name(k) == b"k_bf16_seq_grad"][0]
+    assert res.info == (b.INFO_SATURATED | probe)
+    b.isopo_set_store_format(b.STORE_BF16)
+    res = b.isopo_layer(X, dY, off, A, b.VAR_NORMALISED, 0.0, b.PATH_MATERIALISE)
+    assert res.info == 0
+    K_o = orc.ntk(orc.sequence_gradients(to_f64(X), to_f64(dY), off))
+    assert rel_fro(res.K.cpu().numpy(), K_o) <= TOL
+
+
 def test_format_is_part_of_the_workspace_tag(b):
     X, dY, off, A = _inputs([70, 130, 64], 256, 256, 61)
     ws = b.alloc_workspace(b.BF16, int(off[-1]), 256, 256, 3, b.PATH_MATERIALISE)
