@@ -246,18 +246,15 @@ __global__ void k_mirror_upper(float* __restrict__ K, int B, const float* __rest
 #define ISOPO_COMBINE_IN_FLIGHT 16
 #endif
 constexpr int kCombineInFlight = ISOPO_COMBINE_IN_FLIGHT;  // 16-byte loads a thread has in flight
-// dW = beta dW + sum_i c_i G_i.  One thread per slot (8 elements of every G_i) of the piece-blocked store.
-// kSplit: the slot is 8 bytes in each of the two e4m3 planes, G_i = (hi + lo / 16) / s_i.
-template <bool kSplit>
-__global__ void __launch_bounds__(256) k_bf16_combine(const void* __restrict__ Gv, long long nchunks /* n_pad / 8 */,
+// dW = beta dW + sum_i c_i G_i.  One thread per 16-byte slot (8 elements of every G_i) of the piece-blocked store.
+__global__ void __launch_bounds__(256) k_bf16_combine(const uint4* __restrict__ G, long long nchunks /* n_pad / 8 */,
                                                        int B, int tiles_n, int d_in, int d_out,
-                                                       const float* __restrict__ coeffs, const float* __restrict__ scales,
-                                                       float* __restrict__ dW, float beta,
-                                                       const WsTag* __restrict__ tag_dev, WsTag tag,
+                                                       const float* __restrict__ coeffs, float* __restrict__ dW,
+                                                       float beta, const WsTag* __restrict__ tag_dev, WsTag tag,
                                                        int32_t* __restrict__ info) {
   if (!ws_tag_matches(tag_dev, tag, info)) return;  // another layer's or microbatch's gradients: touch nothing
   __shared__ float sc[256];
-  for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = kSplit ? coeffs[i] / scales[i] : coeffs[i];
+  for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = coeffs[i];
   __syncthreads();
   for (long long pos = blockIdx.x * (long long)blockDim.x + threadIdx.x; pos < nchunks;
        pos += (long long)gridDim.x * blockDim.x) {
@@ -269,61 +266,25 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const void* __restrict__ G
     if (!ISOPO_IN_RANGE((long long)stored_slot((size_t)piece, B - 1, B, l), nchunks * B, info, kIdCombine)) continue;
     if (!ISOPO_IN_RANGE((long long)m * d_in + n + 7, (long long)d_out * d_in, info, kIdCombine)) continue;
     float acc[8] = {};
-    const size_t first = stored_slot((size_t)piece, 0, B, l);
+    const uint4* src = G + stored_slot((size_t)piece, 0, B, l);
     const size_t stride = 32;  // slots between successive sequences of one piece
-    if (kSplit) {
-      const uint2* hi = static_cast<const uint2*>(Gv) + first;
-      const uint2* lo = hi + (size_t)nchunks * B;
-      constexpr int kN = kCombineInFlight / 2;
-      int i = 0;
-      auto add = [&](const uint2& hv, const uint2& lv, float c) {
-        const uint32_t hw[4] = {hv.x & 0xffffu, hv.x >> 16, hv.y & 0xffffu, hv.y >> 16};
-        const uint32_t lw[4] = {lv.x & 0xffffu, lv.x >> 16, lv.y & 0xffffu, lv.y >> 16};
+    auto add = [&](const uint4& v, float c) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int h = 0; h < 4; ++h) {
-          // hi + lo / 16 in half precision is exact (4 + 4 significant bits, at most 9 binades apart)
-          const float2 g = __half22float2(__hfma2(e4m3x2_to_half2(lw[h]), __float2half2_rn(1.f / kLoScale), e4m3x2_to_half2(hw[h])));
-          acc[2 * h] = fmaf(c, g.x, acc[2 * h]);
-          acc[2 * h + 1] = fmaf(c, g.y, acc[2 * h + 1]);
-        }
-      };
-      for (; i + kN <= B; i += kN) {
-        uint2 hv[kN], lv[kN];
-#pragma unroll
-        for (int u = 0; u < kN; ++u) { hv[u] = __ldcs(hi + (size_t)(i + u) * stride); lv[u] = __ldcs(lo + (size_t)(i + u) * stride); }
-#pragma unroll
-        for (int u = 0; u < kN; ++u) add(hv[u], lv[u], sc[i + u]);
+      for (int h = 0; h < 4; ++h) {
+        acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
+        acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
       }
-      for (; i < B; ++i) add(__ldcs(hi + (size_t)i * stride), __ldcs(lo + (size_t)i * stride), sc[i]);
-    } else {
-      const uint4* src = static_cast<const uint4*>(Gv) + first;
-      int i = 0;
-      for (; i + kCombineInFlight <= B; i += kCombineInFlight) {
-        uint4 v[kCombineInFlight];
+    };
+    int i = 0;
+    for (; i + kCombineInFlight <= B; i += kCombineInFlight) {
+      uint4 v[kCombineInFlight];
 #pragma unroll
-        for (int u = 0; u < kCombineInFlight; ++u) v[u] = __ldcs(src + (size_t)(i + u) * stride);
+      for (int u = 0; u < kCombineInFlight; ++u) v[u] = __ldcs(src + (size_t)(i + u) * stride);
 #pragma unroll
-        for (int u = 0; u < kCombineInFlight; ++u) {
-          const float c = sc[i + u];
-          const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-          for (int h = 0; h < 4; ++h) {
-            acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
-            acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
-          }
-        }
-      }
-      for (; i < B; ++i) {
-        const uint4 v = __ldcs(src + (size_t)i * stride);
-        const float c = sc[i];
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int h = 0; h < 4; ++h) {
-          acc[2 * h] = fmaf(c, __uint_as_float(w[h] << 16), acc[2 * h]);
-          acc[2 * h + 1] = fmaf(c, __uint_as_float(w[h] & 0xffff0000u), acc[2 * h + 1]);
-        }
-      }
+      for (int u = 0; u < kCombineInFlight; ++u) add(v[u], sc[i + u]);
     }
+    for (; i < B; ++i) add(__ldcs(src + (size_t)i * stride), sc[i]);
     float4* out = reinterpret_cast<float4*>(dW + (size_t)m * d_in + n);
     float4 o0 = make_float4(acc[0], acc[1], acc[2], acc[3]), o1 = make_float4(acc[4], acc[5], acc[6], acc[7]);
     if (beta != 0.f) {
@@ -333,6 +294,73 @@ __global__ void __launch_bounds__(256) k_bf16_combine(const void* __restrict__ G
     }
     out[0] = o0;
     out[1] = o1;
+  }
+}
+
+// Split store: dW = beta dW + sum_i (c_i / s_i) (hi_i + lo_i / 16).  One thread per PAIR of slots (two tile rows x 8
+// columns), so that every load is 16 bytes per plane: with one slot per thread the two planes cost twice the load
+// instructions per byte of the bf16 store and the pass fell to 5.0 TB/s inside the step.
+__global__ void __launch_bounds__(256) k_e4m3_combine(const uint2* __restrict__ planes, long long nchunks /* n_pad / 8 */,
+                                                       int B, int tiles_n, int d_in, int d_out,
+                                                       const float* __restrict__ coeffs, const float* __restrict__ scales,
+                                                       float* __restrict__ dW, float beta,
+                                                       const WsTag* __restrict__ tag_dev, WsTag tag,
+                                                       int32_t* __restrict__ info) {
+  if (!ws_tag_matches(tag_dev, tag, info)) return;  // another layer's or microbatch's gradients: touch nothing
+  __shared__ float sc[256];
+  for (int i = threadIdx.x; i < B; i += blockDim.x) sc[i] = coeffs[i] / scales[i];
+  __syncthreads();
+  const long long npairs = nchunks / 2;
+  for (long long pos = blockIdx.x * (long long)blockDim.x + threadIdx.x; pos < npairs;
+       pos += (long long)gridDim.x * blockDim.x) {
+    // pos = piece * 16 + pair of slots; piece = (tile * 32 + j) * 4 + q
+    const long long piece = pos >> 4;
+    const int l = (int)(pos & 15) * 2, q = (int)(piece & 3), j = (int)((piece >> 2) & 31), tile = (int)(piece >> 7);
+    const int m = (tile / tiles_n) * kTileM + q * 32 + l, n = (tile % tiles_n) * kTileN + j * 8;
+    if (m >= d_out || n >= d_in) continue;
+    if (!ISOPO_IN_RANGE((long long)stored_slot((size_t)piece, B - 1, B, l + 1), nchunks * B, info, kIdCombine)) continue;
+    if (!ISOPO_IN_RANGE((long long)m * d_in + n + 7, (long long)d_out * d_in, info, kIdCombine)) continue;
+    float acc[16] = {};
+    const uint4* hi = reinterpret_cast<const uint4*>(planes + stored_slot((size_t)piece, 0, B, l));
+    const uint4* lo = reinterpret_cast<const uint4*>(planes + (size_t)nchunks * B + stored_slot((size_t)piece, 0, B, l));
+    const size_t stride = 16;  // 16-byte units between successive sequences of one piece
+    auto add = [&](const uint4& hv, const uint4& lv, float c) {
+      const uint32_t hw[8] = {hv.x & 0xffffu, hv.x >> 16, hv.y & 0xffffu, hv.y >> 16,
+                              hv.z & 0xffffu, hv.z >> 16, hv.w & 0xffffu, hv.w >> 16};
+      const uint32_t lw[8] = {lv.x & 0xffffu, lv.x >> 16, lv.y & 0xffffu, lv.y >> 16,
+                              lv.z & 0xffffu, lv.z >> 16, lv.w & 0xffffu, lv.w >> 16};
+#pragma unroll
+      for (int h = 0; h < 8; ++h) {
+        // hi + lo / 16 in half precision is exact (4 + 4 significant bits, at most 9 binades apart)
+        const float2 g = __half22float2(__hfma2(e4m3x2_to_half2(lw[h]), __float2half2_rn(1.f / kLoScale), e4m3x2_to_half2(hw[h])));
+        acc[2 * h] = fmaf(c, g.x, acc[2 * h]);
+        acc[2 * h + 1] = fmaf(c, g.y, acc[2 * h + 1]);
+      }
+    };
+    constexpr int kN = kCombineInFlight / 2;
+    int i = 0;
+    for (; i + kN <= B; i += kN) {
+      uint4 hv[kN], lv[kN];
+#pragma unroll
+      for (int u = 0; u < kN; ++u) { hv[u] = __ldcs(hi + (size_t)(i + u) * stride); lv[u] = __ldcs(lo + (size_t)(i + u) * stride); }
+#pragma unroll
+      for (int u = 0; u < kN; ++u) add(hv[u], lv[u], sc[i + u]);
+    }
+    for (; i < B; ++i) add(__ldcs(hi + (size_t)i * stride), __ldcs(lo + (size_t)i * stride), sc[i]);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (m + r >= d_out) break;
+      float4* out = reinterpret_cast<float4*>(dW + (size_t)(m + r) * d_in + n);
+      float4 o0 = make_float4(acc[8 * r], acc[8 * r + 1], acc[8 * r + 2], acc[8 * r + 3]);
+      float4 o1 = make_float4(acc[8 * r + 4], acc[8 * r + 5], acc[8 * r + 6], acc[8 * r + 7]);
+      if (beta != 0.f) {
+        const float4 p0 = out[0], p1 = out[1];
+        o0.x += p0.x; o0.y += p0.y; o0.z += p0.z; o0.w += p0.w;
+        o1.x += p1.x; o1.y += p1.y; o1.z += p1.z; o1.w += p1.w;
+      }
+      out[0] = o0;
+      out[1] = o1;
+    }
   }
 }
 
@@ -397,11 +425,11 @@ isopo_status bf16_combine(const void* G, const WsLayout& L, int d_in, int d_out,
   {
     LaunchScope scope(kIdCombine, st);
     if (fmt.split)
-      k_bf16_combine<true><<<grid, 256, 0, st>>>(G, chunks, B, L.tiles_n, d_in, d_out, coeffs, fmt.scales, dW, beta, tag_dev,
-                                                 tag, info);
+      k_e4m3_combine<<<grid, 256, 0, st>>>((const uint2*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, fmt.scales, dW, beta,
+                                           tag_dev, tag, info);
     else
-      k_bf16_combine<false><<<grid, 256, 0, st>>>(G, chunks, B, L.tiles_n, d_in, d_out, coeffs, nullptr, dW, beta, tag_dev,
-                                                  tag, info);
+      k_bf16_combine<<<grid, 256, 0, st>>>((const uint4*)G, chunks, B, L.tiles_n, d_in, d_out, coeffs, dW, beta, tag_dev, tag,
+                                           info);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
