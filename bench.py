@@ -279,6 +279,8 @@ def run_gpu(args):
     variant = b.VAR_INTERACTING if args.variant == "interacting" else b.VAR_NORMALISED
 
     sampled = args.route == "sampled"
+    if args.deterministic:  # before any workspace is sized: the per-CTA partial sums of K live there
+        b.isopo_set_deterministic(True)
     if args.store_format == "e4m3_split":  # before any workspace is sized or written
         b.isopo_set_store_format(b.STORE_E4M3_SPLIT)
     # Algorithm 1 draws its overlap samples with randperm: the bench draws them once, seeded, on the host
@@ -715,7 +717,7 @@ def run_gpu(args):
         "config": {"workload": args.workload, "B": B, "tokens": T,
                    "route": "sampled (Algorithm 1, %d token samples)" % len(sample_rows) if sampled else "stored gradients",
                    "variant": "normalised (Algorithm 1)" if sampled else args.variant,
-                   "store_format": args.store_format,
+                   "store_format": args.store_format, "deterministic": bool(args.deterministic),
                    "layers": cfg_layers, "paths": cfg_paths,
                    "l2": ("L2 flushed between steps (256 MB fill, untimed); every step timed by its own events"
                           if flush else "inputs larger than L2 (no flush needed)"),
@@ -763,6 +765,8 @@ def main():
     ap.add_argument("--schedule", default="batched", choices=["batched", "single"],
                     help="stored route: batched = every projection keeps its workspace and one launch solves for all "
                          "their coefficients; single = one call per projection, one shared workspace")
+    ap.add_argument("--deterministic", action="store_true",
+                    help="stored route: K summed over the CTAs in a fixed order (isopo_set_deterministic)")
     ap.add_argument("--graph", action="store_true",
                     help="also capture one step in a CUDA graph and time its replays (reported under cuda_graph)")
     ap.add_argument("--skip-e2e", action="store_true")
