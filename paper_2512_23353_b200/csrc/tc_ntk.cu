@@ -222,15 +222,27 @@ __global__ void __launch_bounds__(kThreads, 1) k_bf16_ntk(const __grid_constant_
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-// Deterministic mode: K[i][j] = K[j][i] = sum over the CTAs, in CTA order, of their partial entry (min(i,j), max(i,j)).
+// Deterministic mode: K[i][j] = K[j][i] = sum over the CTAs, in CTA order, of their partial entry (i, j), i <= j.
+// One thread per entry of the upper triangle (its reads run along a row of every partial matrix), which also
+// writes the mirrored entry.
 __global__ void k_ntk_reduce(const float* __restrict__ kpart, int n_ctas, int B, float* __restrict__ K) {
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= B * B) return;
   const int i = e / B, j = e % B;
-  const size_t src = (size_t)min(i, j) * B + max(i, j), stride = (size_t)B * B;
+  if (j < i) return;
+  const size_t stride = (size_t)B * B;
   float s = 0.f;
-  for (int c = 0; c < n_ctas; ++c) s += kpart[c * stride + src];
+  int c = 0;
+  for (; c + 8 <= n_ctas; c += 8) {  // eight loads in flight; the additions keep the CTA order
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = __ldcs(kpart + (c + u) * stride + e);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += v[u];
+  }
+  for (; c < n_ctas; ++c) s += __ldcs(kpart + c * stride + e);
   K[e] = s;
+  K[(size_t)j * B + i] = s;
 }
 
 // kdiag != NULL (split store): the diagonal comes from the gradient GEMM's float32 sums of squares
