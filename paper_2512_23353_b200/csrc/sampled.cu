@@ -30,6 +30,38 @@ __device__ __forceinline__ double block_sum_d(double v) {
   return v;
 }
 
+// Copies one token row and returns this thread's share of its sum of squares.  Rows whose byte length and both
+// addresses are multiples of 16 (every bfloat16 layer the library accepts) move as 16-byte vectors.
+template <typename T>
+__device__ __forceinline__ double copy_row_sq(const T* __restrict__ src, T* __restrict__ dst, int d) {
+  constexpr int kVec = 16 / (int)sizeof(T);
+  double acc = 0.0;
+  if (d % kVec == 0 && (((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
+    const uint4* s4 = reinterpret_cast<const uint4*>(src);
+    uint4* d4 = reinterpret_cast<uint4*>(dst);
+    for (int c = threadIdx.x; c < d / kVec; c += blockDim.x) {
+      const uint4 v = __ldg(s4 + c);
+      d4[c] = v;
+      const T* e = reinterpret_cast<const T*>(&v);
+      float part = 0.f;  // at most 8 squares of bfloat16 / 4 of float32 values: exact enough before the float64 sum
+#pragma unroll
+      for (int k = 0; k < kVec; ++k) {
+        const float f = to_f32(e[k]);
+        if (sizeof(T) == 2) part = fmaf(f, f, part); else acc += (double)f * (double)f;
+      }
+      if (sizeof(T) == 2) acc += (double)part;
+    }
+    return acc;
+  }
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const T v = src[c];
+    dst[c] = v;
+    const double f = (double)to_f32(v);
+    acc += f * f;
+  }
+  return acc;
+}
+
 // Block j copies token row rows[j] of X and dY into a0[j], g0[j] and adds ||g0_j||^2 ||a0_j||^2 to *den.
 template <typename T>
 __global__ void __launch_bounds__(256) k_gather_samples(const T* __restrict__ X, const T* __restrict__ dY, int d_in,
@@ -38,19 +70,8 @@ __global__ void __launch_bounds__(256) k_gather_samples(const T* __restrict__ X,
                                                         double* __restrict__ den) {
   const int j = blockIdx.x;
   const int64_t t = rows[j];
-  double na = 0.0, ng = 0.0;
-  for (int c = threadIdx.x; c < d_in; c += blockDim.x) {
-    const T v = X[t * d_in + c];
-    a0[(size_t)j * d_in + c] = v;
-    const double f = (double)to_f32(v);
-    na += f * f;
-  }
-  for (int c = threadIdx.x; c < d_out; c += blockDim.x) {
-    const T v = dY[t * d_out + c];
-    g0[(size_t)j * d_out + c] = v;
-    const double f = (double)to_f32(v);
-    ng += f * f;
-  }
+  double na = copy_row_sq(X + t * d_in, a0 + (size_t)j * d_in, d_in);
+  double ng = copy_row_sq(dY + t * d_out, g0 + (size_t)j * d_out, d_out);
   na = block_sum_d(na);
   ng = block_sum_d(ng);
   if (threadIdx.x == 0) atomicAdd(den, na * ng);
@@ -101,18 +122,30 @@ __global__ void __launch_bounds__(256) k_f32_sampled(const float* __restrict__ X
     }
 }
 
-// F_i^2 = sum_j M^T[j, i]^2 / den,  c_i = A_i / sqrt(F_i^2 + lambda).  One thread per sequence.
+// F_i^2 = sum_j M^T[j, i]^2 / den,  c_i = A_i / sqrt(F_i^2 + lambda).  A block of 32 x 8 threads serves 32
+// sequences: thread (x, y) sums the samples j = y, y + 8, ... of sequence x (loads coalesced over x), the eight
+// partial sums meet in shared memory.
+constexpr int kFinishSlices = 8;
 template <typename TM>
-__global__ void k_sampled_finish(const TM* __restrict__ Mt, int n_samples, int B, const double* __restrict__ den,
-                                 const float* __restrict__ A, float lambda, float* __restrict__ coeffs,
-                                 float* __restrict__ F2) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= B) return;
+__global__ void __launch_bounds__(32 * kFinishSlices) k_sampled_finish(const TM* __restrict__ Mt, int n_samples, int B,
+                                                                       const double* __restrict__ den,
+                                                                       const float* __restrict__ A, float lambda,
+                                                                       float* __restrict__ coeffs, float* __restrict__ F2) {
+  __shared__ double part[kFinishSlices][32];
+  const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
+  const int i = blockIdx.x * 32 + x;
   double s = 0.0;
-  for (int j = 0; j < n_samples; ++j) {
-    const double m = (double)Mt[(size_t)j * B + i];
-    s += m * m;
-  }
+  if (i < B)
+    for (int j = y; j < n_samples; j += kFinishSlices) {
+      const double m = (double)Mt[(size_t)j * B + i];
+      s += m * m;
+    }
+  part[y][x] = s;
+  __syncthreads();
+  if (y != 0 || i >= B) return;
+  s = 0.0;
+#pragma unroll
+  for (int k = 0; k < kFinishSlices; ++k) s += part[k][x];
   const double f2 = s / *den;
   if (F2) F2[i] = (float)f2;
   coeffs[i] = (float)((double)A[i] / sqrt(f2 + (double)lambda));
@@ -167,7 +200,7 @@ isopo_status sampled_coefficients(const void* X, const void* dY, isopo_dtype dty
     ISOPO_CUDA_TRY(cudaGetLastError());
     {
       LaunchScope scope(kIdSampledAux, st);
-      k_sampled_finish<double><<<(B + 127) / 128, 128, 0, st>>>(Mt, n_samples, B, den, A, lambda, coeffs, F2);
+      k_sampled_finish<double><<<(B + 31) / 32, 32 * kFinishSlices, 0, st>>>(Mt, n_samples, B, den, A, lambda, coeffs, F2);
     }
     ISOPO_CUDA_TRY(cudaGetLastError());
     return ISOPO_OK;
@@ -185,7 +218,7 @@ isopo_status sampled_coefficients(const void* X, const void* dY, isopo_dtype dty
   if (s != ISOPO_OK) return s;
   {
     LaunchScope scope(kIdSampledAux, st);
-    k_sampled_finish<float><<<(B + 127) / 128, 128, 0, st>>>(Mt, n_samples, B, den, A, lambda, coeffs, F2);
+    k_sampled_finish<float><<<(B + 31) / 32, 32 * kFinishSlices, 0, st>>>(Mt, n_samples, B, den, A, lambda, coeffs, F2);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;
