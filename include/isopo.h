@@ -202,6 +202,27 @@ ISOPO_API isopo_status isopo_transform_advantages(const float* K, const float* A
                                         const float* opt_pqr_regs, float* coeffs, int32_t* info, void* cuda_stream);
 
 /*
+ * isopo_transform_advantages_large: the interacting variant, (K + lambda I) c = A (Sec. 3 display; Alg. 2), for
+ * up to ISOPO_MAX_LARGE_SEQS sequences.  Same blocked Cholesky and float64-residual refinement as
+ * isopo_transform_advantages, with the block triangle of the factor kept in `workspace` (2.1 MB at 1024
+ * sequences: it stays in the L2) instead of shared memory; one CTA, milliseconds rather than 0.1 ms.  K of more than
+ * 256 sequences comes from the GRAM path of isopo_layer_gram; the simple variants take any B in
+ * isopo_transform_advantages.  A non-positive pivot k (1-based) is reported as *info = k, coeffs are then zero.
+ *
+ *   K          dev, float32 [B, B] row-major, symmetric; 1 <= B <= ISOPO_MAX_LARGE_SEQS
+ *   A, coeffs  dev, float32 [B]
+ *   lambda     absolute regulariser, >= 0
+ *   workspace  dev, 16-byte aligned, at least isopo_transform_large_workspace_bytes(B) bytes (0 for a B out of
+ *              range); scratch, contents undefined afterwards; must not be shared by calls that overlap
+ * Errors: ISOPO_ERR_INVALID_ARG, ISOPO_ERR_UNSUPPORTED (B too large), ISOPO_ERR_WORKSPACE (too small).
+ */
+#define ISOPO_MAX_LARGE_SEQS 1024
+ISOPO_API size_t isopo_transform_large_workspace_bytes(int B);
+ISOPO_API isopo_status isopo_transform_advantages_large(const float* K, const float* A, int B, float lambda, float* coeffs,
+                                                        void* workspace, size_t workspace_bytes, int32_t* info,
+                                                        void* cuda_stream);
+
+/*
  * Relative regularisation (Alg. 1: "use e.g. EMA of trailing minibatch means for the regularization";
  * generalised re-scaling figure: reg(val) = val + regularization * expectation(val); Sec. 4:
  * "regularization factor 1.0 * E[mean(D)] ... EMA over minibatches with 0.9 decay").

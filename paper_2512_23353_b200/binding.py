@@ -36,7 +36,9 @@ EXPORTS = (
     "isopo_spectral_workspace_bytes", "isopo_transform_spectral", "isopo_transform_spectral_batched",
     "isopo_selftest_bounded_wait", "isopo_set_deterministic", "isopo_get_deterministic", "isopo_debug_build",
     "isopo_set_store_format", "isopo_get_store_format",
+    "isopo_transform_large_workspace_bytes", "isopo_transform_advantages_large",
 )
+MAX_LARGE_SEQS = 1024
 MAX_SAMPLES = 4096
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 65536, 256
 NUM_KERNELS = 17
@@ -90,6 +92,11 @@ def _load():
     lib.isopo_sampled_coefficients.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_void_p,
                                                c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_float, c.c_void_p,
                                                c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.isopo_transform_large_workspace_bytes.restype = c.c_size_t
+    lib.isopo_transform_large_workspace_bytes.argtypes = [c.c_int]
+    lib.isopo_transform_advantages_large.restype = c.c_int
+    lib.isopo_transform_advantages_large.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_float, c.c_void_p, c.c_void_p,
+                                                     c.c_size_t, c.c_void_p, c.c_void_p]
     lib.isopo_reg_ema_update.restype = c.c_int
     lib.isopo_reg_ema_update.argtypes = [c.c_void_p, c.c_int, c.c_float, c.c_void_p, c.c_void_p]
     lib.isopo_transform_advantages_batched.restype = c.c_int
@@ -257,6 +264,20 @@ def isopo_transform_advantages(K: torch.Tensor, A: torch.Tensor, variant: int, l
                                         g.ctypes.data if g is not None else None, coeffs.data_ptr(),
                                         info.data_ptr(), _stream())
     _check(st, "isopo_transform_advantages")
+
+
+def isopo_transform_large_workspace_bytes(B: int) -> int:
+    return int(lib.isopo_transform_large_workspace_bytes(B))
+
+
+def isopo_transform_advantages_large(K: torch.Tensor, A: torch.Tensor, lam: float, coeffs: torch.Tensor, ws: torch.Tensor,
+                                     info: torch.Tensor) -> None:
+    B = A.numel()
+    assert K.dtype == torch.float32 and A.dtype == torch.float32 and coeffs.dtype == torch.float32
+    assert K.is_contiguous() and K.numel() == B * B and coeffs.numel() == B and ws.dtype == torch.uint8
+    st = lib.isopo_transform_advantages_large(K.data_ptr(), A.data_ptr(), B, float(lam), coeffs.data_ptr(), ws.data_ptr(),
+                                              ws.numel(), info.data_ptr(), _stream())
+    _check(st, "isopo_transform_advantages_large")
 
 
 def isopo_reg_ema_update(K: torch.Tensor, decay: float, state: torch.Tensor) -> None:

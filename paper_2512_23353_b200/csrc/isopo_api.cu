@@ -403,6 +403,20 @@ isopo_status isopo_transform_advantages(const float* K, const float* A, int B, i
   return transform(K, A, B, variant, lambda, opt_pqr_regs, nullptr, coeffs, info, (cudaStream_t)cuda_stream);
 }
 
+size_t isopo_transform_large_workspace_bytes(int B) {
+  return B >= 1 && B <= ISOPO_MAX_LARGE_SEQS ? transform_large_workspace_bytes(B) : 0;
+}
+
+isopo_status isopo_transform_advantages_large(const float* K, const float* A, int B, float lambda, float* coeffs,
+                                              void* workspace, size_t workspace_bytes, int32_t* info, void* cuda_stream) {
+  ApiRange nvtx_range("isopo_transform_advantages_large");
+  if (!K || !A || !coeffs || !info || !workspace || B < 1) return ISOPO_ERR_INVALID_ARG;
+  if (!(lambda >= 0.0f) || ((uintptr_t)workspace & 15)) return ISOPO_ERR_INVALID_ARG;
+  if (B > ISOPO_MAX_LARGE_SEQS) return ISOPO_ERR_UNSUPPORTED;
+  if (workspace_bytes < transform_large_workspace_bytes(B)) return ISOPO_ERR_WORKSPACE;
+  return transform_large(K, A, B, lambda, coeffs, (float*)workspace, info, (cudaStream_t)cuda_stream);
+}
+
 isopo_status isopo_reg_ema_update(const float* K, int B, float decay, float* state, void* cuda_stream) {
   ApiRange nvtx_range("isopo_reg_ema_update");
   if (!K || !state || B < 1 || !(decay >= 0.0f && decay < 1.0f)) return ISOPO_ERR_INVALID_ARG;

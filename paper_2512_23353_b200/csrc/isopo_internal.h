@@ -214,6 +214,9 @@ isopo_status sampled_coefficients(const void* X, const void* dY, isopo_dtype dty
                                   int32_t* info, cudaStream_t st);
 
 // transform (all variants)
+size_t transform_large_workspace_bytes(int B);
+isopo_status transform_large(const float* K, const float* A, int B, float lambda, float* coeffs, float* scratch,
+                             int32_t* info, cudaStream_t st);
 isopo_status transform(const float* K, const float* A, int B, isopo_variant v, float lambda, const float* pqr_regs_host,
                        const float* rel_state, float* coeffs, int32_t* info, cudaStream_t st);
 isopo_status transform_batched(int n, const float* const* K, const float* A, int B, isopo_variant v, const float* lambda,

@@ -76,10 +76,17 @@ __device__ __forceinline__ float warp_column_sums(float (&r)[kNB]) {
   return r[0];
 }
 
+// Pointer types of the block helpers.  The factor lives either in this CTA's shared memory (no other writer: the
+// pointers may be restrict-qualified) or, for more than 256 sequences, in a workspace that stays in the L2, where a
+// block written by one warp is read by others after a CTA barrier: plain loads only, never the read-only path.
+template <bool kInWorkspace> struct BlkPtr { typedef float* __restrict__ rw; typedef const float* __restrict__ ro; };
+template <> struct BlkPtr<true> { typedef float* rw; typedef const float* ro; };
+
 // Factors the 32 x 32 diagonal block D (column-major, symmetric input) in place into its lower
 // Cholesky factor and writes 1 / L_kk to rd[k].  One warp.
 // Returns 0, or the 1-based local index of the first non-positive pivot.
-__device__ __noinline__ int warp_factor_diag(float* __restrict__ D, float* __restrict__ rd) {
+template <bool kW>
+__device__ __noinline__ int warp_factor_diag(typename BlkPtr<kW>::rw D, float* __restrict__ rd) {
   const int lane = threadIdx.x & 31;
   float r[kNB];
 #pragma unroll
@@ -107,7 +114,8 @@ __device__ __noinline__ int warp_factor_diag(float* __restrict__ D, float* __res
 
 // Inv = L^-1 (column-major) for the factored diagonal block D with rd[k] = 1 / L_kk.  One warp.
 // Column sweep: lane j solves L z = e_j; after step k, z[k] = Inv[k][j] is final.
-__device__ __noinline__ void warp_invert_factor(const float* __restrict__ D, const float* __restrict__ rd,
+template <bool kW>
+__device__ __noinline__ void warp_invert_factor(typename BlkPtr<kW>::ro D, const float* __restrict__ rd,
                                                 float* __restrict__ Inv) {
   const int lane = threadIdx.x & 31;
   float z[kNB];
@@ -125,7 +133,8 @@ __device__ __noinline__ void warp_invert_factor(const float* __restrict__ D, con
 
 // X L^T = A for one 32 x 32 block A (in place); lane owns a row.  L: factored diagonal block,
 // rd[k] = 1 / L_kk.  Column k of X is final after step k and is eliminated from the later columns.
-__device__ __noinline__ void warp_solve_panel(float* __restrict__ A, const float* __restrict__ L,
+template <bool kW>
+__device__ __noinline__ void warp_solve_panel(typename BlkPtr<kW>::rw A, typename BlkPtr<kW>::ro L,
                                               const float* __restrict__ rd) {
   const int lane = threadIdx.x & 31;
   float a[kNB];
@@ -142,8 +151,9 @@ __device__ __noinline__ void warp_solve_panel(float* __restrict__ A, const float
 }
 
 // C -= A * Bm^T for 32 x 32 blocks (all column-major); lane computes a 4 x 8 sub-tile.
-__device__ __noinline__ void warp_rank32_update(float* __restrict__ C, const float* __restrict__ A,
-                                                const float* __restrict__ Bm) {
+template <bool kW>
+__device__ __noinline__ void warp_rank32_update(typename BlkPtr<kW>::rw C, typename BlkPtr<kW>::ro A,
+                                                typename BlkPtr<kW>::ro Bm) {
   const int lane = threadIdx.x & 31, r0 = (lane & 7) * 4, c0 = (lane >> 3) * 8;
   float4 acc[8];
 #pragma unroll
@@ -167,7 +177,8 @@ __device__ __noinline__ void warp_rank32_update(float* __restrict__ C, const flo
 }
 
 // Solves L L^T x = v in place (v in shared memory, nb*32 entries) with the blocked factor.
-__device__ __noinline__ void block_cholesky_solve(const float* __restrict__ Lb, const float* __restrict__ InvD,
+template <bool kW>
+__device__ __noinline__ void block_cholesky_solve(typename BlkPtr<kW>::ro Lb, const float* __restrict__ InvD,
                                                   float* __restrict__ v, int nb) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   // forward: L y = v
@@ -217,6 +228,180 @@ __device__ __noinline__ void block_cholesky_solve(const float* __restrict__ Lb, 
     }
     __syncthreads();
   }
+}
+
+// Interacting variant, (K + lambda I) c = A: blocked Cholesky of the lower block triangle held at Lb (nb(nb+1)/2
+// blocks; shared memory, or the workspace with kW), the inverse diagonal factors at InvD, then the solve and up to
+// two refinement rounds.  Called by every thread of the CTA; `layer` tags a failed pivot in *info.
+template <bool kW>
+__device__ __forceinline__ void interacting_solve(const TransformParams& P, typename BlkPtr<kW>::rw Lb, float* InvD,
+                                                  float* vec, double* sol, float* rdiag, double& s_trace, double& s_res,
+                                                  int& s_fail, int layer) {
+  const int B = P.B, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kThreads / 32;
+  const float* __restrict__ K = P.K;
+  const int nb = (B + kNB - 1) / kNB, Bp = nb * kNB;
+  if (tid == 0) s_fail = 0;
+  // load the lower block triangle.  K is symmetric, so row j of K read along i gives column j of
+  // the blocks; float4 loads, eight in flight per thread, when B is a multiple of 4.
+  if ((B & 3) == 0) {
+    const int nvec = B * B / 4;
+    for (int base = tid; base < nvec; base += kThreads * 8) {
+      float4 val[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + u * kThreads;
+        val[u] = e < nvec ? __ldg(reinterpret_cast<const float4*>(K) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + u * kThreads;
+        if (e >= nvec) continue;
+        const int j = (e * 4) / B, i = (e * 4) % B, I = i / kNB, J = j / kNB;
+        if (I < J) continue;
+        float4 w = val[u];
+        if (i == j) w.x += P.lambda;
+        if (i + 1 == j) w.y += P.lambda;
+        if (i + 2 == j) w.z += P.lambda;
+        if (i + 3 == j) w.w += P.lambda;
+        *reinterpret_cast<float4*>(Lb + blk_slot(I, J) * kBlk + (j % kNB) * kNB + (i % kNB)) = w;
+      }
+    }
+  } else {
+    for (int e = tid; e < B * B; e += kThreads) {
+      const int j = e / B, i = e % B, I = i / kNB, J = j / kNB;
+      if (I >= J) Lb[blk_slot(I, J) * kBlk + (j % kNB) * kNB + (i % kNB)] = K[e] + (i == j ? P.lambda : 0.f);
+    }
+  }
+  // identity padding of the last block row / column
+  for (int e = tid; e < (Bp - B) * Bp; e += kThreads) {
+    const int i = B + e / Bp, j = e % Bp;  // rows B..Bp-1, all columns j <= i
+    if (j <= i || j / kNB == i / kNB)
+      Lb[blk_slot(i / kNB, j / kNB) * kBlk + (j % kNB) * kNB + (i % kNB)] = i == j ? 1.f : 0.f;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int f = warp_factor_diag<kW>(Lb, rdiag);
+    if (f != 0 && lane == 0) s_fail = f;
+  }
+  __syncthreads();
+  for (int J = 0; J < nb && !s_fail; ++J) {
+    const float* Ljj = Lb + blk_slot(J, J) * kBlk;
+    // panel: blocks (I, J) below the diagonal on warps 0 .. nwarps-2; the last warp inverts L_JJ
+    if (warp == nwarps - 1) warp_invert_factor<kW>(Ljj, rdiag + J * kNB, InvD + J * kBlk);
+    else
+      for (int I = J + 1 + warp; I < nb; I += nwarps - 1) warp_solve_panel<kW>(Lb + blk_slot(I, J) * kBlk, Ljj, rdiag + J * kNB);
+    __syncthreads();
+    // trailing blocks (I, Kc) with I >= Kc > J; t = a(a+1)/2 + rem -> I = J+1+a, Kc = J+1+rem.
+    // t = 0 is the next diagonal block: all warps update it together, then warp 0 factors it while the
+    // others work through the rest
+    const int m = nb - 1 - J, ntrail = m * (m + 1) / 2;
+    if (m > 0) {
+      // all warps: rank-32 update of the next diagonal block, kNB / nwarps columns each (lane = row)
+      float* Dn = Lb + blk_slot(J + 1, J + 1) * kBlk;
+      const float* Pn = Lb + blk_slot(J + 1, J) * kBlk;
+      constexpr int kColsPerWarp = kNB / (kThreads / 32);
+      float acc[kColsPerWarp];
+#pragma unroll
+      for (int c = 0; c < kColsPerWarp; ++c) acc[c] = Dn[(warp * kColsPerWarp + c) * kNB + lane];
+#pragma unroll 8
+      for (int p = 0; p < kNB; ++p) {
+        const float a = Pn[p * kNB + lane];
+#pragma unroll
+        for (int c = 0; c < kColsPerWarp; ++c) acc[c] = fmaf(-a, Pn[p * kNB + warp * kColsPerWarp + c], acc[c]);
+      }
+#pragma unroll
+      for (int c = 0; c < kColsPerWarp; ++c) Dn[(warp * kColsPerWarp + c) * kNB + lane] = acc[c];
+      __syncthreads();
+      if (warp == 0) {
+        const int f = warp_factor_diag<kW>(Dn, rdiag + (J + 1) * kNB);
+        if (f != 0 && lane == 0) s_fail = (J + 1) * kNB + f;
+      } else {
+        for (int t = warp; t < ntrail; t += nwarps - 1) {
+          int a = 0, rem = t;
+          while (rem > a) { rem -= a + 1; ++a; }
+          const int I = J + 1 + a, Kc = J + 1 + rem;
+          warp_rank32_update<kW>(Lb + blk_slot(I, Kc) * kBlk, Lb + blk_slot(I, J) * kBlk, Lb + blk_slot(Kc, J) * kBlk);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  __syncthreads();
+  if (s_fail) {
+    if (tid == 0) atomicCAS(P.info, 0, s_fail + (layer << 16));
+    for (int i = tid; i < B; i += kThreads) P.coeffs[i] = 0.f;
+    return;
+  }
+  // solve, then refinement rounds with a float64 residual while it is above float32 round-off
+  double anorm2 = 0.0;
+  for (int i = tid; i < Bp; i += kThreads) {
+    const float a = i < B ? P.A[i] : 0.f;
+    vec[i] = a;
+    sol[i] = 0.0;
+    anorm2 += (double)a * a;
+  }
+  anorm2 = warp_sum(anorm2);
+  if (tid == 0) { s_trace = 0.0; s_res = 0.0; }
+  __syncthreads();
+  if (lane == 0) atomicAdd(&s_trace, anorm2);
+  __syncthreads();
+  anorm2 = s_trace;
+  for (int round = 0; round < 3; ++round) {
+    block_cholesky_solve<kW>(Lb, InvD, vec, nb);
+    for (int i = tid; i < Bp; i += kThreads) sol[i] += (double)vec[i];
+    __syncthreads();
+    if (round == 2) break;
+    double rn2 = 0.0;
+    for (int i0 = warp * 4; i0 < B; i0 += nwarps * 4) {  // four rows per warp pass: independent loads
+      double acc[4] = {0.0, 0.0, 0.0, 0.0};
+      if ((B & 3) == 0) {
+        for (int j0 = lane * 4; j0 < B; j0 += 256) {  // two float4 per lane and row in flight
+          float4 kv[4][2];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int j = j0 + h * 128;
+              kv[u][h] = (i0 + u < B && j < B) ? __ldg(reinterpret_cast<const float4*>(K + (size_t)(i0 + u) * B + j))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int j = j0 + h * 128;
+            if (j >= B) continue;
+            const double s0 = sol[j], s1 = sol[j + 1], s2 = sol[j + 2], s3 = sol[j + 3];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              acc[u] += (double)kv[u][h].x * s0 + (double)kv[u][h].y * s1 + (double)kv[u][h].z * s2 +
+                        (double)kv[u][h].w * s3;
+          }
+        }
+      } else {
+        for (int j = lane; j < B; j += 32) {
+          const double sj = sol[j];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (i0 + u < B) acc[u] += (double)K[(size_t)(i0 + u) * B + j] * sj;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const double a = warp_sum(acc[u]);
+        if (lane == 0 && i0 + u < B) {
+          const double r = (double)P.A[i0 + u] - a - (double)P.lambda * sol[i0 + u];
+          vec[i0 + u] = (float)r;
+          rn2 += r * r;
+        }
+      }
+    }
+    if (lane == 0) atomicAdd(&s_res, rn2);
+    __syncthreads();
+    const bool done = s_res <= 1e-14 * anorm2;  // relative residual below 1e-7
+    __syncthreads();
+    if (tid == 0) s_res = 0.0;
+    if (done) break;
+  }
+  for (int i = tid; i < B; i += kThreads) P.coeffs[i] = (float)sol[i];
 }
 
 __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ TransformBatch batch) {
@@ -297,168 +482,22 @@ __global__ void __launch_bounds__(kThreads) k_transform(const __grid_constant__ 
   float* vec = InvD + (size_t)nb * kBlk;                    // Bp floats
   double* sol = reinterpret_cast<double*>(vec + Bp);        // Bp doubles (8-byte aligned: all counts even)
   float* rdiag = reinterpret_cast<float*>(sol + Bp);        // Bp floats: 1 / L_kk
-  if (tid == 0) s_fail = 0;
-  // load the lower block triangle.  K is symmetric, so row j of K read along i gives column j of
-  // the blocks; float4 loads, eight in flight per thread, when B is a multiple of 4.
-  if ((B & 3) == 0) {
-    const int nvec = B * B / 4;
-    for (int base = tid; base < nvec; base += kThreads * 8) {
-      float4 val[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int e = base + u * kThreads;
-        val[u] = e < nvec ? __ldg(reinterpret_cast<const float4*>(K) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int e = base + u * kThreads;
-        if (e >= nvec) continue;
-        const int j = (e * 4) / B, i = (e * 4) % B, I = i / kNB, J = j / kNB;
-        if (I < J) continue;
-        float4 w = val[u];
-        if (i == j) w.x += P.lambda;
-        if (i + 1 == j) w.y += P.lambda;
-        if (i + 2 == j) w.z += P.lambda;
-        if (i + 3 == j) w.w += P.lambda;
-        *reinterpret_cast<float4*>(Lb + blk_slot(I, J) * kBlk + (j % kNB) * kNB + (i % kNB)) = w;
-      }
-    }
-  } else {
-    for (int e = tid; e < B * B; e += kThreads) {
-      const int j = e / B, i = e % B, I = i / kNB, J = j / kNB;
-      if (I >= J) Lb[blk_slot(I, J) * kBlk + (j % kNB) * kNB + (i % kNB)] = K[e] + (i == j ? P.lambda : 0.f);
-    }
-  }
-  // identity padding of the last block row / column
-  for (int e = tid; e < (Bp - B) * Bp; e += kThreads) {
-    const int i = B + e / Bp, j = e % Bp;  // rows B..Bp-1, all columns j <= i
-    if (j <= i || j / kNB == i / kNB)
-      Lb[blk_slot(i / kNB, j / kNB) * kBlk + (j % kNB) * kNB + (i % kNB)] = i == j ? 1.f : 0.f;
-  }
-  __syncthreads();
-  if (warp == 0) {
-    const int f = warp_factor_diag(Lb, rdiag);
-    if (f != 0 && lane == 0) s_fail = f;
-  }
-  __syncthreads();
-  for (int J = 0; J < nb && !s_fail; ++J) {
-    const float* Ljj = Lb + blk_slot(J, J) * kBlk;
-    // panel: blocks (I, J) below the diagonal on warps 0 .. nwarps-2; the last warp inverts L_JJ
-    if (warp == nwarps - 1) warp_invert_factor(Ljj, rdiag + J * kNB, InvD + J * kBlk);
-    else
-      for (int I = J + 1 + warp; I < nb; I += nwarps - 1) warp_solve_panel(Lb + blk_slot(I, J) * kBlk, Ljj, rdiag + J * kNB);
-    __syncthreads();
-    // trailing blocks (I, Kc) with I >= Kc > J; t = a(a+1)/2 + rem -> I = J+1+a, Kc = J+1+rem.
-    // t = 0 is the next diagonal block: all warps update it together, then warp 0 factors it while the
-    // others work through the rest
-    const int m = nb - 1 - J, ntrail = m * (m + 1) / 2;
-    if (m > 0) {
-      // all warps: rank-32 update of the next diagonal block, kNB / nwarps columns each (lane = row)
-      float* Dn = Lb + blk_slot(J + 1, J + 1) * kBlk;
-      const float* Pn = Lb + blk_slot(J + 1, J) * kBlk;
-      constexpr int kColsPerWarp = kNB / (kThreads / 32);
-      float acc[kColsPerWarp];
-#pragma unroll
-      for (int c = 0; c < kColsPerWarp; ++c) acc[c] = Dn[(warp * kColsPerWarp + c) * kNB + lane];
-#pragma unroll 8
-      for (int p = 0; p < kNB; ++p) {
-        const float a = Pn[p * kNB + lane];
-#pragma unroll
-        for (int c = 0; c < kColsPerWarp; ++c) acc[c] = fmaf(-a, Pn[p * kNB + warp * kColsPerWarp + c], acc[c]);
-      }
-#pragma unroll
-      for (int c = 0; c < kColsPerWarp; ++c) Dn[(warp * kColsPerWarp + c) * kNB + lane] = acc[c];
-      __syncthreads();
-      if (warp == 0) {
-        const int f = warp_factor_diag(Dn, rdiag + (J + 1) * kNB);
-        if (f != 0 && lane == 0) s_fail = (J + 1) * kNB + f;
-      } else {
-        for (int t = warp; t < ntrail; t += nwarps - 1) {
-          int a = 0, rem = t;
-          while (rem > a) { rem -= a + 1; ++a; }
-          const int I = J + 1 + a, Kc = J + 1 + rem;
-          warp_rank32_update(Lb + blk_slot(I, Kc) * kBlk, Lb + blk_slot(I, J) * kBlk, Lb + blk_slot(Kc, J) * kBlk);
-        }
-      }
-    }
-    __syncthreads();
-  }
-  __syncthreads();
-  if (s_fail) {
-    if (tid == 0) atomicCAS(P.info, 0, s_fail + ((int)blockIdx.x << 16));
-    for (int i = tid; i < B; i += kThreads) P.coeffs[i] = 0.f;
-    return;
-  }
-  // solve, then refinement rounds with a float64 residual while it is above float32 round-off
-  double anorm2 = 0.0;
-  for (int i = tid; i < Bp; i += kThreads) {
-    const float a = i < B ? P.A[i] : 0.f;
-    vec[i] = a;
-    sol[i] = 0.0;
-    anorm2 += (double)a * a;
-  }
-  anorm2 = warp_sum(anorm2);
-  if (tid == 0) { s_trace = 0.0; s_res = 0.0; }
-  __syncthreads();
-  if (lane == 0) atomicAdd(&s_trace, anorm2);
-  __syncthreads();
-  anorm2 = s_trace;
-  for (int round = 0; round < 3; ++round) {
-    block_cholesky_solve(Lb, InvD, vec, nb);
-    for (int i = tid; i < Bp; i += kThreads) sol[i] += (double)vec[i];
-    __syncthreads();
-    if (round == 2) break;
-    double rn2 = 0.0;
-    for (int i0 = warp * 4; i0 < B; i0 += nwarps * 4) {  // four rows per warp pass: independent loads
-      double acc[4] = {0.0, 0.0, 0.0, 0.0};
-      if ((B & 3) == 0) {
-        for (int j0 = lane * 4; j0 < B; j0 += 256) {  // two float4 per lane and row in flight
-          float4 kv[4][2];
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const int j = j0 + h * 128;
-              kv[u][h] = (i0 + u < B && j < B) ? __ldg(reinterpret_cast<const float4*>(K + (size_t)(i0 + u) * B + j))
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int j = j0 + h * 128;
-            if (j >= B) continue;
-            const double s0 = sol[j], s1 = sol[j + 1], s2 = sol[j + 2], s3 = sol[j + 3];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-              acc[u] += (double)kv[u][h].x * s0 + (double)kv[u][h].y * s1 + (double)kv[u][h].z * s2 +
-                        (double)kv[u][h].w * s3;
-          }
-        }
-      } else {
-        for (int j = lane; j < B; j += 32) {
-          const double sj = sol[j];
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            if (i0 + u < B) acc[u] += (double)K[(size_t)(i0 + u) * B + j] * sj;
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const double a = warp_sum(acc[u]);
-        if (lane == 0 && i0 + u < B) {
-          const double r = (double)P.A[i0 + u] - a - (double)P.lambda * sol[i0 + u];
-          vec[i0 + u] = (float)r;
-          rn2 += r * r;
-        }
-      }
-    }
-    if (lane == 0) atomicAdd(&s_res, rn2);
-    __syncthreads();
-    const bool done = s_res <= 1e-14 * anorm2;  // relative residual below 1e-7
-    __syncthreads();
-    if (tid == 0) s_res = 0.0;
-    if (done) break;
-  }
-  for (int i = tid; i < B; i += kThreads) P.coeffs[i] = (float)sol[i];
+  interacting_solve<false>(P, Lb, InvD, vec, sol, rdiag, s_trace, s_res, s_fail, (int)blockIdx.x);
+}
+
+// The interacting variant for more sequences than the shared-memory kernel holds: the block triangle (2.1 MB at
+// 1024 sequences) lives in a workspace that stays in the L2, everything else as above.  One CTA.
+constexpr int kMaxLargeB = ISOPO_MAX_LARGE_SEQS;
+__global__ void __launch_bounds__(kThreads) k_transform_large(const TransformParams P, float* scratch) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ double s_trace, s_res;
+  __shared__ int s_fail;
+  const int nb = (P.B + kNB - 1) / kNB, Bp = nb * kNB;
+  float* InvD = reinterpret_cast<float*>(smem_raw);         // nb inverse diagonal factors
+  float* vec = InvD + (size_t)nb * kBlk;                    // Bp floats
+  double* sol = reinterpret_cast<double*>(vec + Bp);        // Bp doubles
+  float* rdiag = reinterpret_cast<float*>(sol + Bp);        // Bp floats
+  interacting_solve<true>(P, scratch, InvD, vec, sol, rdiag, s_trace, s_res, s_fail, 0);
 }
 
 // Running means for the relative regulariser.  state = {E[F^2], E[||G||^2], E[F^2 / ||G||^2], number of updates};
@@ -532,6 +571,27 @@ isopo_status transform_batched(int n, const float* const* K, const float* A, int
   {
     LaunchScope scope(kIdTransform, st);
     k_transform<<<n, kThreads, smem, st>>>(T);
+  }
+  ISOPO_CUDA_TRY(cudaGetLastError());
+  return ISOPO_OK;
+}
+
+size_t transform_large_workspace_bytes(int B) {
+  const size_t nb = (size_t)(B + kNB - 1) / kNB;
+  return sizeof(float) * (nb * (nb + 1) / 2) * kBlk;
+}
+
+isopo_status transform_large(const float* K, const float* A, int B, float lambda, float* coeffs, float* scratch,
+                             int32_t* info, cudaStream_t st) {
+  if (B < 1 || B > kMaxLargeB) return ISOPO_ERR_UNSUPPORTED;
+  TransformParams P{};
+  P.K = K; P.A = A; P.coeffs = coeffs; P.info = info; P.B = B; P.variant = (int)ISOPO_VAR_INTERACTING; P.lambda = lambda;
+  const size_t nb = (size_t)(B + kNB - 1) / kNB;
+  const size_t smem = sizeof(float) * (nb * kBlk + 2 * nb * kNB) + sizeof(double) * nb * kNB;
+  ISOPO_CUDA_TRY(cudaFuncSetAttribute(k_transform_large, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  {
+    LaunchScope scope(kIdTransform, st);
+    k_transform_large<<<1, kThreads, smem, st>>>(P, scratch);
   }
   ISOPO_CUDA_TRY(cudaGetLastError());
   return ISOPO_OK;

@@ -137,6 +137,16 @@ def test_new_entry_points_validate_on_the_host(binding):
         b.isopo_set_deterministic(False)
     assert b.isopo_workspace_bytes(b.BF16, 4096, 1536, 8960, 16, b.PATH_MATERIALISE) == base
     assert not b.isopo_debug_build()
+    # interacting solve for more than 256 sequences: lower block triangle of 32 x 32 float32 blocks in the workspace
+    assert b.isopo_transform_large_workspace_bytes(1024) == 528 * 4096
+    assert b.isopo_transform_large_workspace_bytes(257) == 45 * 4096
+    assert b.isopo_transform_large_workspace_bytes(0) == 0 and b.isopo_transform_large_workspace_bytes(1025) == 0
+    large = lambda **kw: b.lib.isopo_transform_advantages_large(  # noqa: E731
+        fake, fake, kw.get("B", 300), kw.get("lam", 0.1), fake, kw.get("ws", fake), kw.get("n", 1 << 22), fake, None)
+    assert large(B=0) == b.ERR_INVALID_ARG and large(lam=-1.0) == b.ERR_INVALID_ARG
+    assert large(ws=None) == b.ERR_INVALID_ARG and large(ws=fake + 4) == b.ERR_INVALID_ARG
+    assert large(B=1025) == b.ERR_UNSUPPORTED
+    assert large(n=55 * 4096 - 1) == b.ERR_WORKSPACE                    # 300 sequences: 10 block rows, 55 blocks
 
 
 def test_binding_has_no_fallback():
