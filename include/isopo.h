@@ -191,7 +191,8 @@ ISOPO_API isopo_status isopo_layer_gram_shared_x_stored(const void* X, int n_pro
  * with g = opt_pqr_regs = {p, q, r, reg_F, reg_G, reg_rel} (host, 6 floats; required for GENERAL,
  * ignored otherwise; `lambda` is ignored for GENERAL).  ISOPO_VAR_INTERACTING factors K + lambda*I
  * by Cholesky in shared memory (float32) and refines the solution with float64 residuals; it
- * requires B <= 256 and reports a non-positive pivot k (1-based) as *info = k.
+ * requires B <= 256 (isopo_transform_advantages_large takes up to 1024) and reports a non-positive pivot k
+ * (1-based) as *info = k.
  *
  *   K       dev, float32 [B, B] row-major (as written by isopo_layer_gram)
  *   A       dev, float32 [B]
