@@ -689,6 +689,42 @@ def run_gpu(args):
         finally:
             b.isopo_set_store_format(b.STORE_BF16)
 
+    # ---- the stored route with ONE workspace reused by every projection (what a backward pass with little spare
+    #      memory does: gram, transform, weight gradient per layer; seven single solves instead of one batched) ----
+    if batched and w.dtype == "bf16" and world == 1 and not args.skip_routes and args.store_format == "bf16":
+        one_ws = aligned(max(ws_sizes))
+
+        def one_ws_step():
+            for L in layers:
+                b.isopo_layer_gram(L["X"], L["dY"], off, L["K"], one_ws, info, L["path"])
+                b.isopo_transform_advantages(L["K"], A, variant, L["lam"], L["c"], info)
+                b.isopo_weight_grad(L["X"], L["dY"], L["c"], off, L["dW"], one_ws, info, L["path"], 0.0)
+
+        for _ in range(3):
+            one_ws_step()
+        torch.cuda.synchronize()
+        n_s = max(1, min(args.steps, 10))
+        o_sampler = ClockSampler(local)
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        o_sampler.start()
+        a.record()
+        for _ in range(n_s):
+            one_ws_step()
+        c.record()
+        torch.cuda.synchronize()
+        o_clocks = o_sampler.stop()
+        if int(info.item()) != 0:
+            raise SystemExit(f"device-side error with one workspace: info={int(info.item()):#x}")
+        o_ms = a.elapsed_time(c) / n_s
+        routes = routes or {}
+        routes["stored_one_workspace"] = {
+            "what": "the stored route with one workspace reused by every projection and a transform launch per "
+                    "projection (the headline step keeps all workspaces and solves the block in one launch); same inputs, same run",
+            "ms_per_step": o_ms, "steps": n_s, "tokens_per_s": T / (o_ms * 1e-3), "overhead_vs_plain_dw_gemm": o_ms / plain_ms,
+            "workspace_gb": max(ws_sizes) / 1e9, "headline_workspaces_gb": sum(ws_sizes) / 1e9, "clocks": o_clocks}
+        del one_ws
+
     # ---- the oracle on this machine's host cores, bounded sample ----
     cpu = None
     if world == 1 and not args.skip_cpu:
