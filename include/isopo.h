@@ -113,7 +113,8 @@ ISOPO_API isopo_path isopo_choose_path(isopo_dtype dtype, int64_t T, int d_in, i
  * materialised path, all B per-sequence gradients (bf16 for ISOPO_BF16, float32 for ISOPO_F32)
  * in a piece-blocked order private to the library; on the bf16 Gram path, the per-token-scaled
  * copy of the narrower of X and dY that isopo_weight_grad feeds to its GEMM
- * (2 * T * min(d_in, d_out) bytes).  It must be 1024-byte aligned.  Returns 0 for invalid sizes.
+ * (2 * T * min(d_in, d_out) bytes).  It must be 1024-byte aligned (cudaMalloc promises 256 bytes only: allocate
+ * 1024 bytes more and round the pointer up).  Returns 0 for invalid sizes.
  */
 ISOPO_API size_t isopo_workspace_bytes(isopo_dtype dtype, int64_t T, int d_in, int d_out, int B, isopo_path path);
 
