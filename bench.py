@@ -510,6 +510,19 @@ def run_gpu(args):
         return total, by_layer
 
     plain_ms, plain_by_layer = block_loop(lambda L: torch.matmul(L["dY"].t(), L["X"]))
+    # for comparison only: one layer at a time, each in a loop of its own (see the note above)
+    plain_isolated_ms = 0.0
+    for L in layers:
+        for _ in range(3):
+            torch.matmul(L["dY"].t(), L["X"])
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            torch.matmul(L["dY"].t(), L["X"])
+        c.record()
+        torch.cuda.synchronize()
+        plain_isolated_ms += a.elapsed_time(c) / args.steps
     # the library's own plain GEMM: isopo_weight_grad on the GEMM route with every coefficient one
     # (bf16 workloads; the ratio above is quoted against the faster of the two, which is cuBLAS)
     own_plain_ms = None
@@ -780,6 +793,7 @@ def run_gpu(args):
         "pct_bf16_peak_sustained": step_tflops / peaks["bf16_tflops_sustained"],
         "plain_dw_gemm_ms": plain_ms,
         "plain_dw_gemm_timing": "the block's GEMMs back to back, steps x block, one pair of events (as the step is timed)",
+        "plain_dw_gemm_per_layer_loops_ms": plain_isolated_ms,
         "plain_dw_gemm_own_ms": own_plain_ms,
         "overhead_vs_plain_dw_gemm": overhead,
         "kernels": kernels,
